@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the CAKE prefill-time eviction path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 4] [--impl reference]
+
+One step = one pass of the whole hot path over one batch of synthetic input:
+for every layer score -> allocate -> evict, then one gather-compaction.  Prints
+one JSON line.  The path does not shard: with N > 1 (torchrun) every rank runs
+an independent replica on its own GPU ("replicas only") and the value is the
+sum of tokens over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "CAKE score+evict+compact prompt tokens/s"
+UNIT = "tokens/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", type=int, default=4, help="config index 1..5 (4 = 128K Llama-3.1-8B shape)")
+    ap.add_argument("--impl", default="cake", choices=["cake", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-layers", type=int, default=1)
+    return ap.parse_args()
+
+
+# ----------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-i", str(self.index), "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            p = [x.strip() for x in ln.split(",")]
+            if len(p) < 6:
+                continue
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, p[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------ CPU oracle leg
+def oracle_sample(w, sample_layers: int):
+    """Times the oracle, as it stands, on `sample_layers` full layers of the
+    workload's first request (score, budgets, top-k, compaction) and scales
+    to all layers.  Returns (tokens/s, seconds, threads, description)."""
+    import numpy as np
+    import torch
+    from oracle import cake_oracle as O
+    from paper_2503_12491_b200 import synth
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    N = w.seq_lens[0]
+    qs, ks, vs = [], [], []
+    w1 = synth.scaled(w, seq_lens=(N,))
+    for l in range(sample_layers):
+        q, k, v = synth.layer_inputs(w1, l, "cpu")
+        qs.append(q[0].float().numpy().astype(np.float64))
+        ks.append(k.float().numpy().astype(np.float64))
+        vs.append(v.float().numpy().astype(np.float64))
+    t0 = time.perf_counter()
+    scored = [O.score_layer(q, k, gamma=w.gamma, pool_kernel=w.pool_kernel, tau1=w.tau1, tau2=w.tau2)
+              for q, k in zip(qs, ks)]
+    # the sampled layers stand for all L: they share the budget the full cascade would give them
+    share = w.total_budget * sample_layers // w.n_layers
+    c = O.cascade([s["indicator"] for s in scored], [s["P"] for s in scored],
+                  total_budget=share, window=w.window, seq_len=N)
+    for l in range(sample_layers):
+        O.compact(ks[l], vs[l], c.positions[l])
+    dt = time.perf_counter() - t0
+    full = dt * w.n_layers / sample_layers * (w.total_tokens / N)
+    desc = (f"{sample_layers} of {w.n_layers} layers of request 0 (N={N}), all steps, float64 NumPy; "
+            f"time scaled by L/{sample_layers}" + (f" and by total/N tokens" if w.total_tokens != N else ""))
+    return w.total_tokens / full, dt, threads, desc
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for _ in range(max(1, args.warmup)):
+        oracle_sample(w, args.cpu_sample_layers)
+    desc = threads = None
+    t_all = 0.0
+    for _ in range(args.steps):
+        v, dt, threads, desc = oracle_sample(w, args.cpu_sample_layers)
+        vals.append(v); t_all += dt
+    value = sum(vals) / len(vals)
+    ms = w.total_tokens / value * 1e3
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w):
+    return {"workload": w.name, "n_layers": w.n_layers, "n_q_heads": w.n_q_heads,
+            "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "seq_lens": list(w.seq_lens),
+            "window": w.window, "pool_kernel": w.pool_kernel, "gamma": w.gamma,
+            "total_budget": w.total_budget, "compaction": "deferred (one gather after the last stage)",
+            "l2": "inputs larger than L2 (every layer's K exceeds 126 MB or the step streams > 1 GB)",
+            "parallelism": "replicas only"}
+
+
+# --------------------------------------------------------------- CUDA leg
+def main():
+    args = parse_args()
+    from paper_2503_12491_b200 import synth
+    w = synth.workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2503_12491_b200 import harness, binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) if os.path.exists(
+            os.path.join(ROOT, "MEASURED_PEAKS.json")) else open(os.devnull) as f:
+        try:
+            peaks = json.load(f)
+        except Exception:
+            peaks = {}
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_kind = "measured" if "hbm_gbs" in peaks else "fallback"
+
+    qs, ks, vs = harness.device_inputs(w)
+    cake = harness.cake_for(w)
+    rows = None
+    L = w.n_layers
+    esize = 4 if w.dtype == "fp32" else 2
+
+    def step(bufs):
+        cake.begin(w.cu_seqlens)
+        for l in range(L):
+            cake.score_layer(l, qs[l], ks[l])
+            cake.allocate(l)
+            cake.evict(l)
+        return cake.compact(ks, vs, k_out=bufs[0], v_out=bufs[1], row_offsets=bufs[2], positions=bufs[3])
+
+    cake.begin(w.cu_seqlens)
+    rows = cake.packed_rows_bound()
+    bufs = (torch.empty(rows, w.head_dim, dtype=w.torch_dtype, device="cuda"),
+            torch.empty(rows, w.head_dim, dtype=w.torch_dtype, device="cuda"),
+            torch.empty(len(w.seq_lens) * L + 1, dtype=torch.int64, device="cuda"),
+            torch.empty(rows, dtype=torch.int32, device="cuda"))
+
+    for _ in range(max(3, args.warmup)):
+        step(bufs)
+    barrier()
+    if cake.status() != 0:
+        raise RuntimeError(f"device status {cake.status()}")
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = binding.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        step(bufs)
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    launches = binding.launch_count() - launches0
+    # second pass of the same K steps with every stage bracketed by CUDA events on the
+    # launching stream: gives the per-kernel durations (the brackets cost a little, so the
+    # headline value comes from the first pass)
+    cake.profile_enable(True)
+    cake.profile_read()
+    evp0, evp1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    evp0.record()
+    for _ in range(args.steps):
+        step(bufs)
+    evp1.record()
+    prof = cake.profile_read()
+    ms_profiled = evp0.elapsed_time(evp1) / args.steps
+    cake.profile_enable(False)
+    clocks = sampler.stop() if rank == 0 else None
+    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    tokens = w.total_tokens * world
+    value = tokens / (ms_step * 1e-3)
+
+    retained_rows = int(bufs[2][-1].item())
+    k_bytes = L * w.n_kv_heads * w.total_tokens * w.head_dim * esize
+    q_bytes = L * len(w.seq_lens) * w.n_q_heads * w.window * w.head_dim * esize
+    out_bytes = 2 * retained_rows * w.head_dim * esize
+    ideal = k_bytes + q_bytes + out_bytes
+
+    # dominant kernel: the window-score pass with the larger share of the step;
+    # algorithmic bytes per launch = one layer's K read once + its window Q
+    phase_ms = {k: v["ms"] / args.steps for k, v in prof.items()}
+    dom = max(("score_rows", "score_cols"), key=lambda k: prof[k]["ms"])
+    dom_ms = prof[dom]["ms"] / max(prof[dom]["spans"], 1)
+    per_launch_bytes = (k_bytes + q_bytes) / L
+    achieved = per_launch_bytes / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else None
+    step_gbps = ideal / (ms_step * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak,
+                "unit": "GB/s", "frac": (achieved / hbm_peak) if achieved else None,
+                "peak_kind": f"{peak_kind} copy bandwidth", "traffic": None,
+                "bytes_per_launch": per_launch_bytes, "ms_per_launch": dom_ms,
+                "launches_timed": prof[dom]["spans"],
+                "phase_ms_per_step": phase_ms, "ms_per_step_with_brackets": ms_profiled,
+                "whole_step": {"ideal_bytes": ideal, "GBps": step_gbps,
+                               "frac_of_measured_peak": step_gbps / hbm_peak,
+                               "frac_of_8TBps_nominal": step_gbps / 8000.0}}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
+            "data": "synthetic", "config": workload_config(w), "gpu_launches": launches,
+            "roofline": roofline, "clocks": clocks}
+
+    # ---- end to end: host-resident Q/K/V, copies inside the timed region
+    if not args.no_e2e:
+        line["e2e"] = e2e_leg(args, w, cake, qs, ks, vs, bufs, world, barrier)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, dt, threads, desc = oracle_sample(w, args.cpu_sample_layers)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": desc, "sample_seconds": dt}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    cake.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def e2e_leg(args, w, cake, qs, ks, vs, bufs, world, barrier):
+    """Same step with Q/K/V in pinned host memory: every layer's tensors are
+    copied host->device inside the timed region (double-buffered against the
+    scoring of the previous layer) and the packed cache is read back."""
+    import torch
+    L = w.n_layers
+    hq = [q.cpu().pin_memory() for q in qs]
+    hk = [k.cpu().pin_memory() for k in ks]
+    hv = [v.cpu().pin_memory() for v in vs]
+    del qs[:]
+    # the gather needs every layer's K/V on the device: reuse the resident tensors as the landing zone
+    rows = bufs[0].shape[0]
+    out_k = torch.empty(bufs[0].shape, dtype=bufs[0].dtype).pin_memory()
+    out_v = torch.empty(bufs[1].shape, dtype=bufs[1].dtype).pin_memory()
+    out_off = torch.empty(bufs[2].shape, dtype=torch.int64).pin_memory()
+    out_pos = torch.empty(bufs[3].shape, dtype=torch.int32).pin_memory()
+    dq = [torch.empty_like(hq[0], device="cuda") for _ in range(L)]
+    arrived = [torch.cuda.Event() for _ in range(L)]
+    copy_stream = torch.cuda.Stream()
+    main = torch.cuda.current_stream()
+
+    def step():
+        cake.begin(w.cu_seqlens)
+        copy_stream.wait_stream(main)              # previous step's gather has read K/V
+        for l in range(L):
+            with torch.cuda.stream(copy_stream):
+                dq[l].copy_(hq[l], non_blocking=True)
+                ks[l].copy_(hk[l], non_blocking=True)
+                vs[l].copy_(hv[l], non_blocking=True)
+                arrived[l].record(copy_stream)
+            main.wait_event(arrived[l])
+            cake.score_layer(l, dq[l], ks[l])
+            cake.allocate(l)
+            cake.evict(l)
+        cake.compact(ks, vs, k_out=bufs[0], v_out=bufs[1], row_offsets=bufs[2], positions=bufs[3])
+        out_off.copy_(bufs[2], non_blocking=True)
+        main.synchronize()
+        n = int(out_off[-1])
+        out_k[:n].copy_(bufs[0][:n], non_blocking=True)
+        out_v[:n].copy_(bufs[1][:n], non_blocking=True)
+        out_pos[:n].copy_(bufs[3][:n], non_blocking=True)
+        main.synchronize()
+        return n
+
+    steps = max(1, min(args.steps, 3))
+    step()
+    barrier()
+    t0 = time.perf_counter()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(steps):
+        n = step()
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1) / steps
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    esize = 4 if w.dtype == "fp32" else 2
+    h2d = sum(x.numel() * x.element_size() for x in hq + hk + hv)
+    d2h = 2 * n * w.head_dim * esize + n * 4 + out_off.numel() * 8
+    return {"value": w.total_tokens * world / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+            "steps": steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "note": "Q/K/V pinned on the host, copied per layer on a side stream; packed cache read back"}
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,193 @@
+/*
+ * libcake -- CAKE prefill-time KV-cache eviction for NVIDIA B200 (sm_100a).
+ *
+ * Cascading and adaptive KV-cache eviction with layer preferences
+ * (arXiv 2503.12491).  For every layer the library scores the observation-window
+ * queries against all prompt keys, turns the window attention into the layer's
+ * preference score and the per-token eviction indicator, re-splits the total
+ * cache budget over the layers seen so far, shrinks every seen layer to its
+ * budget with a per-head top-k on the stored indicators, and finally gathers
+ * the retained K/V rows into a packed variable-length cache.
+ *
+ * Conventions
+ *   - Every function returns an int32_t status: CAKE_OK (0) or a negative
+ *     CAKE_ERR_* code.  Nothing throws, exits or prints.
+ *   - Unless a parameter says "host", tensor pointers are DEVICE pointers that
+ *     the caller owns and keeps alive until the stream has consumed them.  The
+ *     context owns only its own state and scratch (allocated in cake_create).
+ *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work;
+ *     none synchronises with the device except cake_status, cake_destroy and
+ *     the *_host convenience entry points, which say so.
+ *   - A context serves one batch of requests at a time and is not thread-safe.
+ *
+ * Shapes: L layers, H_q query heads, H_kv KV heads, G = H_q/H_kv, d = head_dim,
+ * request r has N_r prompt tokens, S_w window queries, n_r = N_r - S_w
+ * non-window tokens, T = sum_r N_r.
+ *
+ * Packed varlen layout of K and V of one layer: [H_kv][T][d], request r owns
+ * token rows cu_seqlens[r] .. cu_seqlens[r+1]-1 of every head.
+ */
+#ifndef CAKE_H_
+#define CAKE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CAKE_OK               0
+#define CAKE_ERR_ARG        (-1)  /* null pointer, bad shape, unsupported size           */
+#define CAKE_ERR_BUDGET     (-2)  /* total_budget < n_layers * window                    */
+#define CAKE_ERR_CAPACITY   (-3)  /* batch exceeds max_requests / max_total_tokens       */
+#define CAKE_ERR_NONFINITE  (-4)  /* a preference is NaN, infinite or negative (device)  */
+#define CAKE_ERR_TIMEOUT    (-5)  /* a bounded device-side wait ran out (device)         */
+#define CAKE_ERR_CUDA       (-6)  /* a CUDA runtime call failed                          */
+#define CAKE_ERR_STATE      (-7)  /* call out of order (layer / stage sequence)          */
+
+#define CAKE_DTYPE_FP32 0
+#define CAKE_DTYPE_BF16 1
+#define CAKE_POOL_MAX   0
+#define CAKE_POOL_AVG   1
+
+#define CAKE_MAX_LAYERS 128
+
+typedef struct cake_ctx cake_ctx;
+
+typedef struct cake_config {
+  int32_t n_layers;         /* L, 1..CAKE_MAX_LAYERS                                      */
+  int32_t n_q_heads;        /* H_q                                                        */
+  int32_t n_kv_heads;       /* H_kv, divides H_q                                          */
+  int32_t head_dim;         /* d: 64 or 128                                               */
+  int32_t window;           /* S_w >= 1; G * S_w <= 128                                   */
+  int32_t pool_kernel;      /* odd, >= 1 (1 = no pooling)                                 */
+  int32_t pool_mode;        /* CAKE_POOL_MAX (window clipped at the ends) or CAKE_POOL_AVG
+                               (zero padding, divisor pool_kernel)                        */
+  int32_t var_ddof;         /* 0 = population variance (default), 1 = unbiased            */
+  int32_t dtype;            /* CAKE_DTYPE_FP32 or CAKE_DTYPE_BF16: element type of Q/K/V  */
+  float   gamma;            /* weight of the variance term in the indicator (Eq. 11)      */
+  float   tau1, tau2;       /* temperatures of the preference score (Eq. 6), > 0          */
+  int64_t total_budget;     /* B_total per request: tokens per KV head summed over layers,
+                               window included; must be >= n_layers * window              */
+  int32_t max_requests;     /* capacity: requests per batch                               */
+  int64_t max_total_tokens; /* capacity: T = sum of prompt lengths per batch              */
+} cake_config;
+
+/* Allocates a context (device state and scratch sized from the capacities) on
+ * the current device.  The only entry point that allocates device memory. */
+int32_t cake_create(const cake_config* cfg, cake_ctx** out);
+/* Synchronises the device and frees everything the context owns. */
+int32_t cake_destroy(cake_ctx* ctx);
+
+/* Starts a new batch and resets the cascade (Algorithm 1, line 1).
+ * cu_seqlens_host: HOST array [n_req+1], exclusive prefix sums of the prompt
+ * lengths, cu[0] = 0; copied before the call returns.  Every N_r >= window.
+ * n_req = 0 is a valid empty batch. */
+int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu_seqlens_host, void* stream);
+
+/* Layer `layer` arrives (Algorithm 1, lines 3-6; Section 2 Eq. 2, Section 3
+ * Eq. 4-5, Section 4.1 Eq. 6, Section 4.3 Eq. 11).  Layers come in order 0..L-1,
+ * each after the previous layer's cake_evict.
+ *   q_win [n_req][H_q][S_w][d]  the last S_w queries of every request
+ *   k     [H_kv][T][d]          packed varlen keys of this layer
+ *   lse   optional [n_req][H_q][S_w] fp32: natural-log sum-exp of each window
+ *         row's scaled logits over its visible keys (as a fused attention
+ *         forward produces); NULL = computed here.
+ * Computes A = softmax(q k^T / sqrt(d)) for the window rows with the causal
+ * mask inside the window, keeps the columns of the n_r non-window keys without
+ * renormalising, and stores in the context
+ *   - the pooled indicator pool1d(Mean_i + gamma Var_i) of the attention
+ *     averaged over each KV head's G query heads,
+ *   - H_l, V_l (means over query heads of the row-entropy sum and of the
+ *     column-variance sum) and P_l = H_l^(1/tau1) V_l^(1/tau2).
+ * Non-finite or negative P_l sets the sticky device status CAKE_ERR_NONFINITE. */
+int32_t cake_score_layer(cake_ctx* ctx, int32_t layer, const void* q_win, const void* k,
+                         const float* lse, void* stream);
+
+/* Budgets of layers 0..stage from the preferences known so far (Section 4.1
+ * Eq. 7, Section 4.2 Eq. 9; Algorithm 1 line 7), entirely on the device.
+ * Each layer owns S_w window slots; the remaining B' = B_total - L*S_w slots
+ * are split in proportion to P_l and integerised by Webster / Sainte-Lague
+ * highest averages (priorities P_l/(s+1/2), IEEE double; ties to the lower
+ * layer, then the lower s), then capped at n_r.  A request with
+ * N_r <= floor(B_total/L) keeps every token.  All-zero preferences count as
+ * all-equal. */
+int32_t cake_allocate(cake_ctx* ctx, int32_t stage, void* stream);
+
+/* Shrinks every layer 0..stage to its current budget (Algorithm 1, lines 9-13;
+ * Section 4.2 EVICT; Section 4.3 Eq. 12): per KV head keeps the entries that
+ * come first in the order (indicator descending, token position ascending)
+ * among the stored (indicator, position) pairs; survivors keep their stored
+ * indicator.  The window tokens are always kept.  Needs cake_allocate(stage)
+ * and stages in order. */
+int32_t cake_evict(cake_ctx* ctx, int32_t stage, void* stream);
+
+/* Gathers the retained rows of layers [layer_lo, layer_hi) (Eq. 12: K^ = K[D,:],
+ * V^ = V[D,:]) into the packed cache.  All of those layers must have been
+ * evicted.
+ *   k_layers, v_layers  HOST arrays [n_layers] of device pointers, each
+ *                       [H_kv][T][d]; entries outside [layer_lo, layer_hi) are ignored
+ *   k_out, v_out        device, capacity >= cake_packed_rows_bound() rows of d elements
+ *   row_offsets_out     device int64 [n_req*L + 1]: block (r,l) = index r*L+l occupies
+ *                       rows row_offsets[r*L+l] .. row_offsets[r*L+l+1]-1 and is laid
+ *                       out [H_kv][len][d], len = its retained length; rows are in
+ *                       ascending token position, the window last
+ *   positions_out       device int32, one token position per packed row (may be NULL) */
+int32_t cake_compact(cake_ctx* ctx, int32_t layer_lo, int32_t layer_hi,
+                     const void* const* k_layers, const void* const* v_layers,
+                     void* k_out, void* v_out, int64_t* row_offsets_out,
+                     int32_t* positions_out, void* stream);
+
+/* Upper bound on the rows cake_compact writes for the current batch:
+ * H_kv * sum_r min(B_total, L*N_r).  Returns the bound or a negative error. */
+int64_t cake_packed_rows_bound(const cake_ctx* ctx);
+
+/* ---- getters (results stay on the device) and test hooks ---------------- */
+
+/* Pooled indicators of the most recently scored (or set) layer, valid until
+ * the next cake_score_layer: out is device fp32 [H_kv][T]; window positions
+ * hold +inf (the paper's "arbitrarily large" value, Section 4.3). */
+int32_t cake_get_indicators(cake_ctx* ctx, int32_t layer, float* out, void* stream);
+/* H, V, P: device double [n_req][L] each (any may be NULL). */
+int32_t cake_get_preferences(cake_ctx* ctx, double* H, double* V, double* P, void* stream);
+/* Retained length of every layer including the window: device int32 [n_req][L];
+ * layers beyond the last allocated stage read 0. */
+int32_t cake_get_budgets(cake_ctx* ctx, int32_t* out, void* stream);
+/* Retained positions of one (request, layer): device int32 [H_kv][len], len as
+ * cake_get_budgets reports; `capacity` = elements available in out. */
+int32_t cake_get_positions(cake_ctx* ctx, int32_t req, int32_t layer, int32_t* out,
+                           int64_t capacity, void* stream);
+/* Replaces cake_score_layer's indicator output for `layer`: in is device fp32
+ * [H_kv][T] (window positions ignored).  Lets a test run the cascade on
+ * indicators computed elsewhere. */
+int32_t cake_set_indicators(cake_ctx* ctx, int32_t layer, const float* in, void* stream);
+/* Sets P for layers 0..n_layers_set-1: device double [n_req][n_layers_set]. */
+int32_t cake_set_preferences(cake_ctx* ctx, int32_t n_layers_set, const double* P, void* stream);
+/* Synchronises `stream`, then returns the sticky device status word through
+ * device_status_out (CAKE_OK or the first CAKE_ERR_* a kernel raised). */
+int32_t cake_status(cake_ctx* ctx, int32_t* device_status_out, void* stream);
+
+/* ---- tracing ------------------------------------------------------------ */
+#define CAKE_PROF_SCORE_ROWS  0  /* window scores, pass A: row max / sum (softmax denominators) */
+#define CAKE_PROF_SCORE_COLS  1  /* window scores, pass B: column statistics -> raw indicator   */
+#define CAKE_PROF_FINALIZE    2  /* preference + pooling                                         */
+#define CAKE_PROF_ALLOCATE    3
+#define CAKE_PROF_EVICT       4
+#define CAKE_PROF_COMPACT     5
+#define CAKE_PROF_KINDS       6
+/* While enabled, every stage of the path brackets its kernels with CUDA events
+ * on the caller's stream (this perturbs back-to-back launches slightly). */
+int32_t cake_profile_enable(cake_ctx* ctx, int32_t on);
+/* Synchronises `stream`; returns, per CAKE_PROF_* kind, the milliseconds and
+ * the number of bracketed spans accumulated since the last read (HOST arrays
+ * of CAKE_PROF_KINDS entries), then clears them. */
+int32_t cake_profile_read(cake_ctx* ctx, double* ms_out, int64_t* spans_out, void* stream);
+
+const char* cake_strerror(int32_t code);
+/* Number of kernels this library has launched in the calling process. */
+int64_t cake_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAKE_H_ */

@@ -1,0 +1,424 @@
+// C-ABI of libcake: context life cycle, the call-order state machine, getters
+// and test hooks.  Every step of the path runs in the kernels of the other
+// translation units; this file only validates arguments and enqueues work.
+#include "cake_internal.cuh"
+
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+namespace cake {
+
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int64_t n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int prof_begin(cake_ctx* ctx, int kind, cudaStream_t st) {
+  Profiler& p = ctx->prof;
+  if (!p.on || p.used >= p.cap) return -1;
+  ProfSpan& s = p.spans[p.used];
+  if (!s.a) {
+    if (cudaEventCreate(&s.a) != cudaSuccess || cudaEventCreate(&s.b) != cudaSuccess) return -1;
+  }
+  s.kind = kind;
+  cudaEventRecord(s.a, st);
+  return p.used++;
+}
+
+void prof_end(cake_ctx* ctx, int span, cudaStream_t st) {
+  if (span >= 0) cudaEventRecord(ctx->prof.spans[span].b, st);
+}
+
+namespace {
+
+template <typename T>
+cudaError_t dev_alloc(T** p, size_t count) {
+  *p = nullptr;
+  if (count == 0) count = 1;
+  return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
+}
+
+int32_t choose_unit_keys(int64_t total_tokens, int n_kv_heads, int n_sm) {
+  // Aim for about four CTAs per SM across the (unit, KV head) grid, units of 64..1024 keys.
+  int64_t per = total_tokens * n_kv_heads / ((int64_t)4 * n_sm);
+  per = per / kSimtTileKeys * kSimtTileKeys;
+  if (per < kSimtTileKeys) per = kSimtTileKeys;
+  if (per > 1024) per = 1024;
+  return (int32_t)per;
+}
+
+__global__ void budgets_with_window(const int32_t* __restrict__ b, int32_t* __restrict__ out,
+                                    int n_req, int L, int n_alloc, int Sw) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_req * L) return;
+  const int l = i % L;
+  out[i] = l < n_alloc ? b[i] + Sw : 0;
+}
+
+void free_ctx(cake_ctx* c) {
+  if (!c) return;
+  cudaFree(c->d_req); cudaFree(c->d_units); cudaFree(c->d_H); cudaFree(c->d_V); cudaFree(c->d_P);
+  cudaFree(c->d_budget[0]); cudaFree(c->d_budget[1]); cudaFree(c->d_status); cudaFree(c->d_raw);
+  cudaFree(c->d_fresh); cudaFree(c->list_vals); cudaFree(c->list_pos); cudaFree(c->d_lse2);
+  cudaFree(c->d_rowpart); cudaFree(c->d_colpart);
+  if (c->h_req) cudaFreeHost(c->h_req);
+  if (c->h_units) cudaFreeHost(c->h_units);
+  if (c->upload_done) cudaEventDestroy(c->upload_done);
+  if (c->prof.spans) {
+    for (int i = 0; i < c->prof.cap; ++i) {
+      if (c->prof.spans[i].a) cudaEventDestroy(c->prof.spans[i].a);
+      if (c->prof.spans[i].b) cudaEventDestroy(c->prof.spans[i].b);
+    }
+    free(c->prof.spans);
+  }
+  free(c->h_cu);
+  delete c;
+}
+
+}  // namespace
+}  // namespace cake
+
+using namespace cake;
+
+extern "C" {
+
+int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
+  if (!cfg || !out) return CAKE_ERR_ARG;
+  *out = nullptr;
+  const cake_config& c = *cfg;
+  if (c.n_layers < 1 || c.n_layers > CAKE_MAX_LAYERS) return CAKE_ERR_ARG;
+  if (c.n_kv_heads < 1 || c.n_q_heads < c.n_kv_heads || c.n_q_heads % c.n_kv_heads) return CAKE_ERR_ARG;
+  if (c.head_dim != 64 && c.head_dim != 128) return CAKE_ERR_ARG;
+  const int G = c.n_q_heads / c.n_kv_heads;
+  if (c.window < 1 || G > 8 || (int64_t)G * c.window > kMaxRows) return CAKE_ERR_ARG;
+  if (c.pool_kernel < 1 || c.pool_kernel % 2 == 0) return CAKE_ERR_ARG;
+  if (c.pool_mode != CAKE_POOL_MAX && c.pool_mode != CAKE_POOL_AVG) return CAKE_ERR_ARG;
+  if (c.var_ddof != 0 && !(c.var_ddof == 1 && c.window >= 2)) return CAKE_ERR_ARG;
+  if (c.dtype != CAKE_DTYPE_FP32 && c.dtype != CAKE_DTYPE_BF16) return CAKE_ERR_ARG;
+  if (!(c.tau1 > 0.f) || !(c.tau2 > 0.f) || !std::isfinite(c.gamma)) return CAKE_ERR_ARG;
+  if (c.max_requests < 1 || c.max_total_tokens < 1) return CAKE_ERR_ARG;
+  if (c.max_total_tokens > ((int64_t)1 << 31) - 1024) return CAKE_ERR_ARG;
+  if (c.total_budget < (int64_t)c.n_layers * c.window) return CAKE_ERR_BUDGET;
+  if (c.total_budget > ((int64_t)1 << 31) - 1024) return CAKE_ERR_ARG;
+
+  cake_ctx* x = new (std::nothrow) cake_ctx();
+  if (!x) return CAKE_ERR_CUDA;
+  memset(x, 0, sizeof(*x));
+  x->cfg = c;
+  x->rows = G * c.window;
+  x->sel_budget = c.total_budget - (int64_t)c.n_layers * c.window;
+  x->alloc_of_buf[0] = x->alloc_of_buf[1] = -1;
+  x->last_alloc = -1;
+  cudaError_t e = cudaGetDevice(&x->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&x->n_sm, cudaDevAttrMultiProcessorCount, x->device);
+  if (e != cudaSuccess) { free_ctx(x); return CAKE_ERR_CUDA; }
+
+  const int64_t T = c.max_total_tokens;
+  const int64_t R = c.max_requests;
+  // a unit never spans requests: at most T/64 + R units
+  x->max_units = (int32_t)(T / kSimtTileKeys + R + 1);
+  int64_t list_tokens = R * x->sel_budget < T ? R * x->sel_budget : T;
+  x->list_elems = list_tokens * c.n_layers * c.n_kv_heads;
+  x->h_cu = (int64_t*)calloc((size_t)R + 1, sizeof(int64_t));
+  bool ok = x->h_cu != nullptr;
+  ok = ok && cudaMallocHost((void**)&x->h_req, sizeof(ReqInfo) * R) == cudaSuccess;
+  ok = ok && cudaMallocHost((void**)&x->h_units, sizeof(ScoreUnit) * x->max_units) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&x->upload_done, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_req, R) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_units, x->max_units) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_H, R * c.n_layers) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_V, R * c.n_layers) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_P, R * c.n_layers) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_budget[0], R * c.n_layers) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_budget[1], R * c.n_layers) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_status, 1) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_raw, (size_t)c.n_kv_heads * T) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_fresh, (size_t)c.n_kv_heads * T) == cudaSuccess;
+  ok = ok && dev_alloc(&x->list_vals, (size_t)x->list_elems) == cudaSuccess;
+  ok = ok && dev_alloc(&x->list_pos, (size_t)x->list_elems) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_lse2, (size_t)R * c.n_q_heads * c.window) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_rowpart, (size_t)x->max_units * c.n_kv_heads * x->rows) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_colpart, (size_t)x->max_units * c.n_kv_heads * G * 2) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_status, 0, sizeof(int32_t)) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_budget[0], 0, sizeof(int32_t) * R * c.n_layers) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_budget[1], 0, sizeof(int32_t) * R * c.n_layers) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_P, 0, sizeof(double) * R * c.n_layers) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_H, 0, sizeof(double) * R * c.n_layers) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_V, 0, sizeof(double) * R * c.n_layers) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); free_ctx(x); return CAKE_ERR_CUDA; }
+  x->n_req = -1;                                  // no batch yet
+  *out = x;
+  return CAKE_OK;
+}
+
+int32_t cake_destroy(cake_ctx* ctx) {
+  if (!ctx) return CAKE_ERR_ARG;
+  cudaError_t e = cudaDeviceSynchronize();
+  free_ctx(ctx);
+  return cuda_status(e);
+}
+
+int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream) {
+  if (!ctx || n_req < 0 || (n_req > 0 && !cu)) return CAKE_ERR_ARG;
+  const cake_config& c = ctx->cfg;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (n_req > c.max_requests) return CAKE_ERR_CAPACITY;
+  if (n_req > 0) {
+    if (cu[0] != 0) return CAKE_ERR_ARG;
+    for (int r = 0; r < n_req; ++r)
+      if (cu[r + 1] - cu[r] < c.window) return CAKE_ERR_ARG;
+    if (cu[n_req] > c.max_total_tokens) return CAKE_ERR_CAPACITY;
+  }
+  const int64_t T = n_req > 0 ? cu[n_req] : 0;
+  const bool same = ctx->n_req == n_req && n_req > 0 &&
+                    memcmp(ctx->h_cu, cu, sizeof(int64_t) * (n_req + 1)) == 0;
+  if (!same && n_req > 0) {
+    if (ctx->upload_pending) {                    // staging buffers still feed an earlier copy
+      CAKE_CUDA_TRY(cudaEventSynchronize(ctx->upload_done));
+      ctx->upload_pending = false;
+    }
+    const int32_t unit_keys = choose_unit_keys(T, c.n_kv_heads, ctx->n_sm);
+    int32_t nu = 0;
+    int64_t list_off = 0, bound = 0;
+    for (int r = 0; r < n_req; ++r) {
+      ReqInfo& q = ctx->h_req[r];
+      q.cu = cu[r];
+      q.N = (int32_t)(cu[r + 1] - cu[r]);
+      q.n = q.N - c.window;
+      q.keep_all = q.N <= c.total_budget / c.n_layers ? 1 : 0;
+      q.cap = (int32_t)(ctx->sel_budget < q.n ? ctx->sel_budget : q.n);
+      q.list_off = list_off;
+      list_off += (int64_t)q.cap * c.n_layers * c.n_kv_heads;
+      q.unit0 = nu;
+      for (int32_t k0 = 0; k0 < q.N; k0 += unit_keys) {
+        ScoreUnit& u = ctx->h_units[nu++];
+        u.req = r; u.key0 = k0; u.nkeys = q.N - k0 < unit_keys ? q.N - k0 : unit_keys; u.pad = 0;
+      }
+      q.nunits = nu - q.unit0;
+      const int64_t full = (int64_t)c.n_layers * q.N;
+      bound += (int64_t)c.n_kv_heads * (c.total_budget < full ? c.total_budget : full);
+    }
+    if (list_off > ctx->list_elems || nu > ctx->max_units) return CAKE_ERR_CAPACITY;
+    ctx->n_units = nu;
+    ctx->packed_rows_bound = bound;
+    memcpy(ctx->h_cu, cu, sizeof(int64_t) * (n_req + 1));
+    CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_req, ctx->h_req, sizeof(ReqInfo) * n_req,
+                                  cudaMemcpyHostToDevice, st));
+    CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_units, ctx->h_units, sizeof(ScoreUnit) * nu,
+                                  cudaMemcpyHostToDevice, st));
+    CAKE_CUDA_TRY(cudaEventRecord(ctx->upload_done, st));
+    ctx->upload_pending = true;
+  }
+  if (n_req == 0) { ctx->n_units = 0; ctx->packed_rows_bound = 0; }
+  ctx->n_req = n_req;
+  ctx->total_tokens = T;
+  ctx->n_ind = ctx->n_pref = ctx->n_evicted = 0;
+  ctx->alloc_of_buf[0] = ctx->alloc_of_buf[1] = -1;
+  ctx->last_alloc = -1;
+  CAKE_CUDA_TRY(cudaMemsetAsync(ctx->d_status, 0, sizeof(int32_t), st));
+  return CAKE_OK;
+}
+
+int32_t cake_score_layer(cake_ctx* ctx, int32_t layer, const void* q_win, const void* k,
+                         const float* lse, void* stream) {
+  if (!ctx || ctx->n_req < 0) return ctx ? CAKE_ERR_STATE : CAKE_ERR_ARG;
+  if (layer < 0 || layer >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
+  if (ctx->n_req > 0 && (!q_win || !k)) return CAKE_ERR_ARG;
+  if (layer != ctx->n_ind || ctx->n_evicted != layer) return CAKE_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t rc = launch_score_simt(ctx, q_win, k, lse, st);
+  if (rc != CAKE_OK) return rc;
+  const int sp = prof_begin(ctx, CAKE_PROF_FINALIZE, st);
+  rc = launch_finalize_layer(ctx, layer, st);
+  if (rc != CAKE_OK) return rc;
+  rc = launch_pool(ctx, st);
+  prof_end(ctx, sp, st);
+  if (rc != CAKE_OK) return rc;
+  ctx->n_ind = layer + 1;
+  if (ctx->n_pref < layer + 1) ctx->n_pref = layer + 1;
+  return CAKE_OK;
+}
+
+int32_t cake_allocate(cake_ctx* ctx, int32_t stage, void* stream) {
+  if (!ctx || ctx->n_req < 0) return ctx ? CAKE_ERR_STATE : CAKE_ERR_ARG;
+  if (stage < 0 || stage >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
+  if (stage >= ctx->n_pref) return CAKE_ERR_STATE;
+  const int sp = prof_begin(ctx, CAKE_PROF_ALLOCATE, (cudaStream_t)stream);
+  int32_t rc = launch_allocate(ctx, stage, (cudaStream_t)stream);
+  prof_end(ctx, sp, (cudaStream_t)stream);
+  if (rc != CAKE_OK) return rc;
+  ctx->alloc_of_buf[stage & 1] = stage;
+  ctx->last_alloc = stage;
+  return CAKE_OK;
+}
+
+int32_t cake_evict(cake_ctx* ctx, int32_t stage, void* stream) {
+  if (!ctx || ctx->n_req < 0) return ctx ? CAKE_ERR_STATE : CAKE_ERR_ARG;
+  if (stage < 0 || stage >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
+  if (stage != ctx->n_evicted || ctx->n_ind != stage + 1) return CAKE_ERR_STATE;
+  if (ctx->alloc_of_buf[stage & 1] != stage) return CAKE_ERR_STATE;
+  if (stage > 0 && ctx->alloc_of_buf[(stage + 1) & 1] != stage - 1) return CAKE_ERR_STATE;
+  const int sp = prof_begin(ctx, CAKE_PROF_EVICT, (cudaStream_t)stream);
+  int32_t rc = launch_evict(ctx, stage, (cudaStream_t)stream);
+  prof_end(ctx, sp, (cudaStream_t)stream);
+  if (rc != CAKE_OK) return rc;
+  ctx->n_evicted = stage + 1;
+  return CAKE_OK;
+}
+
+int32_t cake_compact(cake_ctx* ctx, int32_t layer_lo, int32_t layer_hi, const void* const* k_layers,
+                     const void* const* v_layers, void* k_out, void* v_out,
+                     int64_t* row_offsets_out, int32_t* positions_out, void* stream) {
+  if (!ctx || ctx->n_req < 0) return ctx ? CAKE_ERR_STATE : CAKE_ERR_ARG;
+  if (layer_lo < 0 || layer_hi > ctx->cfg.n_layers || layer_lo > layer_hi) return CAKE_ERR_ARG;
+  if (!row_offsets_out) return CAKE_ERR_ARG;
+  if (layer_hi > ctx->n_evicted || ctx->n_evicted < 1) return CAKE_ERR_STATE;
+  if (ctx->last_alloc != ctx->n_evicted - 1) return CAKE_ERR_STATE;
+  LayerPtrs ptrs;
+  memset(&ptrs, 0, sizeof(ptrs));
+  if (ctx->n_req > 0 && layer_hi > layer_lo) {
+    if (!k_layers || !v_layers || !k_out || !v_out) return CAKE_ERR_ARG;
+    for (int l = layer_lo; l < layer_hi; ++l) {
+      if (!k_layers[l] || !v_layers[l]) return CAKE_ERR_ARG;
+      ptrs.k[l] = k_layers[l];
+      ptrs.v[l] = v_layers[l];
+    }
+  }
+  const int sp = prof_begin(ctx, CAKE_PROF_COMPACT, (cudaStream_t)stream);
+  const int32_t rc = launch_compact(ctx, layer_lo, layer_hi, ptrs, k_out, v_out, row_offsets_out,
+                                    positions_out, (cudaStream_t)stream);
+  prof_end(ctx, sp, (cudaStream_t)stream);
+  return rc;
+}
+
+int64_t cake_packed_rows_bound(const cake_ctx* ctx) {
+  if (!ctx) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0) return CAKE_ERR_STATE;
+  return ctx->packed_rows_bound;
+}
+
+int32_t cake_get_indicators(cake_ctx* ctx, int32_t layer, float* out, void* stream) {
+  if (!ctx || !out) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0 || layer != ctx->n_ind - 1) return CAKE_ERR_STATE;
+  if (ctx->total_tokens == 0) return CAKE_OK;
+  CAKE_CUDA_TRY(cudaMemcpyAsync(out, ctx->d_fresh,
+                                sizeof(float) * ctx->cfg.n_kv_heads * ctx->total_tokens,
+                                cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return CAKE_OK;
+}
+
+int32_t cake_get_preferences(cake_ctx* ctx, double* H, double* V, double* P, void* stream) {
+  if (!ctx) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0) return CAKE_ERR_STATE;
+  const size_t bytes = sizeof(double) * ctx->n_req * ctx->cfg.n_layers;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (bytes == 0) return CAKE_OK;
+  if (H) CAKE_CUDA_TRY(cudaMemcpyAsync(H, ctx->d_H, bytes, cudaMemcpyDeviceToDevice, st));
+  if (V) CAKE_CUDA_TRY(cudaMemcpyAsync(V, ctx->d_V, bytes, cudaMemcpyDeviceToDevice, st));
+  if (P) CAKE_CUDA_TRY(cudaMemcpyAsync(P, ctx->d_P, bytes, cudaMemcpyDeviceToDevice, st));
+  return CAKE_OK;
+}
+
+int32_t cake_set_indicators(cake_ctx* ctx, int32_t layer, const float* in, void* stream) {
+  if (!ctx || !in) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0) return CAKE_ERR_STATE;
+  if (layer < 0 || layer >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
+  if (layer != ctx->n_ind || ctx->n_evicted != layer) return CAKE_ERR_STATE;
+  if (ctx->total_tokens > 0)
+    CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_fresh, in,
+                                  sizeof(float) * ctx->cfg.n_kv_heads * ctx->total_tokens,
+                                  cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  ctx->n_ind = layer + 1;
+  return CAKE_OK;
+}
+
+int32_t cake_set_preferences(cake_ctx* ctx, int32_t n_set, const double* P, void* stream) {
+  if (!ctx || !P) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0) return CAKE_ERR_STATE;
+  if (n_set < 1 || n_set > ctx->cfg.n_layers) return CAKE_ERR_ARG;
+  if (ctx->n_req > 0)
+    CAKE_CUDA_TRY(cudaMemcpy2DAsync(ctx->d_P, sizeof(double) * ctx->cfg.n_layers, P,
+                                    sizeof(double) * n_set, sizeof(double) * n_set, ctx->n_req,
+                                    cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  if (ctx->n_pref < n_set) ctx->n_pref = n_set;
+  return CAKE_OK;
+}
+
+int32_t cake_get_budgets(cake_ctx* ctx, int32_t* out, void* stream) {
+  if (!ctx || !out) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0 || ctx->last_alloc < 0) return CAKE_ERR_STATE;
+  if (ctx->n_req == 0) return CAKE_OK;
+  const int total = ctx->n_req * ctx->cfg.n_layers;
+  budgets_with_window<<<(total + 127) / 128, 128, 0, (cudaStream_t)stream>>>(
+      ctx->d_budget[ctx->last_alloc & 1], out, ctx->n_req, ctx->cfg.n_layers, ctx->last_alloc + 1,
+      ctx->cfg.window);
+  count_launch();
+  return cuda_status(cudaGetLastError());
+}
+
+int32_t cake_get_positions(cake_ctx* ctx, int32_t req, int32_t layer, int32_t* out, int64_t capacity,
+                           void* stream) {
+  if (!ctx || !out || capacity < 0) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0) return CAKE_ERR_STATE;
+  if (req < 0 || req >= ctx->n_req || layer < 0 || layer >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
+  if (layer >= ctx->n_evicted || ctx->last_alloc != ctx->n_evicted - 1) return CAKE_ERR_STATE;
+  return launch_get_positions(ctx, req, layer, out, capacity, (cudaStream_t)stream);
+}
+
+int32_t cake_status(cake_ctx* ctx, int32_t* device_status_out, void* stream) {
+  if (!ctx) return CAKE_ERR_ARG;
+  int32_t s = 0;
+  cudaStream_t st = (cudaStream_t)stream;
+  CAKE_CUDA_TRY(cudaMemcpyAsync(&s, ctx->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  CAKE_CUDA_TRY(cudaStreamSynchronize(st));
+  if (device_status_out) *device_status_out = s;
+  return CAKE_OK;
+}
+
+int32_t cake_profile_enable(cake_ctx* ctx, int32_t on) {
+  if (!ctx) return CAKE_ERR_ARG;
+  Profiler& p = ctx->prof;
+  if (on && !p.spans) {
+    p.cap = 16384;
+    p.spans = (ProfSpan*)calloc(p.cap, sizeof(ProfSpan));
+    if (!p.spans) { p.cap = 0; return CAKE_ERR_CUDA; }
+  }
+  p.on = on != 0;
+  return CAKE_OK;
+}
+
+int32_t cake_profile_read(cake_ctx* ctx, double* ms_out, int64_t* spans_out, void* stream) {
+  if (!ctx || !ms_out || !spans_out) return CAKE_ERR_ARG;
+  CAKE_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+  for (int k = 0; k < CAKE_PROF_KINDS; ++k) { ms_out[k] = 0.0; spans_out[k] = 0; }
+  Profiler& p = ctx->prof;
+  for (int i = 0; i < p.used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, p.spans[i].a, p.spans[i].b) == cudaSuccess) {
+      ms_out[p.spans[i].kind] += ms;
+      spans_out[p.spans[i].kind] += 1;
+    }
+  }
+  p.used = 0;
+  cudaGetLastError();
+  return CAKE_OK;
+}
+
+const char* cake_strerror(int32_t code) {
+  switch (code) {
+    case CAKE_OK: return "ok";
+    case CAKE_ERR_ARG: return "invalid argument";
+    case CAKE_ERR_BUDGET: return "total budget smaller than n_layers * window";
+    case CAKE_ERR_CAPACITY: return "batch exceeds the context's capacity";
+    case CAKE_ERR_NONFINITE: return "non-finite or negative preference";
+    case CAKE_ERR_TIMEOUT: return "device-side wait timed out";
+    case CAKE_ERR_CUDA: return "CUDA runtime error";
+    case CAKE_ERR_STATE: return "call out of order";
+    default: return "unknown error";
+  }
+}
+
+int64_t cake_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

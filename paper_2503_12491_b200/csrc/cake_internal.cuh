@@ -1,0 +1,124 @@
+// Internal declarations shared by the translation units of libcake.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "cake.h"
+
+namespace cake {
+
+constexpr int kMaxRows = 128;        // G * S_w rows handled per KV head
+constexpr int kSimtTileKeys = 64;    // keys per tile of the SIMT score kernels
+constexpr int kSimtThreads = 256;
+
+// One request of the current batch (device copy in ctx->d_req).
+struct ReqInfo {
+  int64_t cu;        // first token row of the request inside the packed K/V
+  int32_t N;         // prompt length
+  int32_t n;         // N - S_w non-window tokens
+  int32_t keep_all;  // 1: N <= floor(B_total/L), nothing is evicted
+  int32_t cap;       // capacity of each (layer, head) list = min(B', n)
+  int64_t list_off;  // first element of this request's lists in list_vals / list_pos
+  int32_t unit0;     // first score unit of the request
+  int32_t nunits;    // number of score units of the request
+};
+
+// A run of consecutive keys of one request handled by one CTA of a score kernel.
+struct ScoreUnit {
+  int32_t req;
+  int32_t key0;
+  int32_t nkeys;
+  int32_t pad;
+};
+
+struct LayerPtrs {
+  const void* k[CAKE_MAX_LAYERS];
+  const void* v[CAKE_MAX_LAYERS];
+};
+
+}  // namespace cake
+
+namespace cake {
+struct ProfSpan { int kind; cudaEvent_t a, b; };
+struct Profiler {
+  bool on;
+  int used, cap;
+  ProfSpan* spans;
+};
+}  // namespace cake
+
+struct cake_ctx {
+  cake_config cfg;
+  cake::Profiler prof;
+  int device;
+  int n_sm;
+  int32_t rows;            // R = G * S_w
+  int64_t sel_budget;      // B' = B_total - L * S_w
+  // ---- batch state (host) ----
+  int32_t n_req;
+  int64_t total_tokens;    // T
+  int32_t n_units;         // score units for all N keys (phase A)
+  int32_t n_ind;           // layers whose indicators have arrived
+  int32_t n_pref;          // layers whose preference is known
+  int32_t n_evicted;       // stages completed
+  int32_t alloc_of_buf[2]; // stage whose budgets live in budget buffer 0/1 (-1 none)
+  int32_t last_alloc;      // most recent stage passed to cake_allocate
+  int64_t packed_rows_bound;
+  int64_t* h_cu;           // host copy of cu_seqlens [max_requests+1]
+  // ---- pinned staging ----
+  cake::ReqInfo* h_req;    // [max_requests]
+  cake::ScoreUnit* h_units;
+  cudaEvent_t upload_done;
+  bool upload_pending;
+  // ---- device state ----
+  cake::ReqInfo* d_req;
+  cake::ScoreUnit* d_units;
+  int32_t max_units;
+  double* d_H;             // [max_requests][L]
+  double* d_V;
+  double* d_P;
+  int32_t* d_budget[2];    // [max_requests][L] selectable budgets, double-buffered by stage parity
+  int32_t* d_status;       // sticky device status word
+  float* d_raw;            // [H_kv][max_total_tokens] un-pooled indicator
+  float* d_fresh;          // [H_kv][max_total_tokens] pooled indicator of the newest layer
+  float* list_vals;        // per (req, layer, head) surviving indicators
+  int32_t* list_pos;       //                        and their token positions
+  int64_t list_elems;
+  float* d_lse2;           // [max_requests][H_q][S_w] base-2 log-sum-exp of window rows
+  float2* d_rowpart;       // [max_units][H_kv][R] (max, sum) partials of phase A
+  float* d_colpart;        // [max_units][H_kv][G][2] partial (sum p*log2 p, sum var) of phase B
+};
+
+namespace cake {
+
+void count_launch(int64_t n = 1);
+
+// score_simt.cu
+int32_t launch_score_simt(cake_ctx* ctx, const void* q_win, const void* k, const float* lse,
+                          cudaStream_t st);
+// cascade.cu
+int32_t launch_finalize_layer(cake_ctx* ctx, int32_t layer, cudaStream_t st);
+int32_t launch_pool(cake_ctx* ctx, cudaStream_t st);
+int32_t launch_allocate(cake_ctx* ctx, int32_t stage, cudaStream_t st);
+int32_t launch_evict(cake_ctx* ctx, int32_t stage, cudaStream_t st);
+// compact.cu
+int32_t launch_compact(cake_ctx* ctx, int32_t lo, int32_t hi, const LayerPtrs& ptrs, void* k_out,
+                       void* v_out, int64_t* row_offsets, int32_t* positions, cudaStream_t st);
+int32_t launch_get_positions(cake_ctx* ctx, int32_t req, int32_t layer, int32_t* out,
+                             int64_t capacity, cudaStream_t st);
+
+// Tracing spans (no-ops unless cake_profile_enable was called).
+int prof_begin(cake_ctx* ctx, int kind, cudaStream_t st);
+void prof_end(cake_ctx* ctx, int span, cudaStream_t st);
+
+inline int32_t cuda_status(cudaError_t e) { return e == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA; }
+
+#define CAKE_CUDA_TRY(expr)                         \
+  do {                                              \
+    cudaError_t _e = (expr);                        \
+    if (_e != cudaSuccess) return CAKE_ERR_CUDA;    \
+  } while (0)
+
+}  // namespace cake
