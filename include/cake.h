@@ -183,6 +183,11 @@ int32_t cake_profile_enable(cake_ctx* ctx, int32_t on);
  * of CAKE_PROF_KINDS entries), then clears them. */
 int32_t cake_profile_read(cake_ctx* ctx, double* ms_out, int64_t* spans_out, void* stream);
 
+/* 1 if cake_score_layer runs the tcgen05 tensor-core kernels for this context
+ * (bf16, G*S_w a multiple of 32 up to 128, G in {1,2,4,8}), 0 if it runs the fp32
+ * SIMT kernels, negative on error. */
+int32_t cake_uses_tensor_cores(const cake_ctx* ctx);
+
 const char* cake_strerror(int32_t code);
 /* Number of kernels this library has launched in the calling process. */
 int64_t cake_launch_count(void);

@@ -28,7 +28,7 @@ EXPORTS = [
     "cake_evict", "cake_compact", "cake_packed_rows_bound", "cake_get_indicators",
     "cake_get_preferences", "cake_get_budgets", "cake_get_positions", "cake_set_indicators",
     "cake_set_preferences", "cake_status", "cake_strerror", "cake_launch_count",
-    "cake_profile_enable", "cake_profile_read",
+    "cake_profile_enable", "cake_profile_read", "cake_uses_tensor_cores",
 ]
 PROF_KINDS = ["score_rows", "score_cols", "finalize", "allocate", "evict", "compact"]
 
@@ -83,6 +83,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.cake_status.argtypes = [vp, ctypes.POINTER(i32), vp]
     lib.cake_profile_enable.argtypes = [vp, i32]
     lib.cake_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64), vp]
+    lib.cake_uses_tensor_cores.argtypes = [vp]
     lib.cake_strerror.argtypes = [i32]
     lib.cake_strerror.restype = ctypes.c_char_p
     lib.cake_launch_count.argtypes = []
@@ -246,6 +247,9 @@ class Cake:
         s = ctypes.c_int32(0)
         _check(self.lib.cake_status(self._h, ctypes.byref(s), _stream()), "cake_status")
         return int(s.value)
+
+    def uses_tensor_cores(self) -> bool:
+        return int(self.lib.cake_uses_tensor_cores(self._h)) == 1
 
     def profile_enable(self, on: bool) -> None:
         _check(self.lib.cake_profile_enable(self._h, 1 if on else 0), "cake_profile_enable")

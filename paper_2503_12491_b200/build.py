@@ -16,7 +16,7 @@ CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG, "libcake.so")
 
-SOURCES = ["cake_api.cu", "score_simt.cu", "cascade.cu", "compact.cu"]
+SOURCES = ["cake_api.cu", "score_simt.cu", "score_tc.cu", "cascade.cu", "compact.cu"]
 
 
 def _nvcc() -> str:

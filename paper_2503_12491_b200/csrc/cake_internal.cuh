@@ -33,6 +33,15 @@ struct ScoreUnit {
   int32_t pad;
 };
 
+// A run of consecutive keys of one (request, KV head) handled by one CTA of the
+// tensor-core score kernels.
+struct TcSegment {
+  int32_t req;
+  int32_t g;
+  int32_t key0;
+  int32_t nkeys;
+};
+
 struct LayerPtrs {
   const void* k[CAKE_MAX_LAYERS];
   const void* v[CAKE_MAX_LAYERS];
@@ -89,6 +98,18 @@ struct cake_ctx {
   float* d_lse2;           // [max_requests][H_q][S_w] base-2 log-sum-exp of window rows
   float2* d_rowpart;       // [max_units][H_kv][R] (max, sum) partials of phase A
   float* d_colpart;        // [max_units][H_kv][G][2] partial (sum p*log2 p, sum var) of phase B
+  // ---- tensor-core score path ----
+  bool use_tc;
+  bool hhead_from_rows;    // entropy came from pass A (d_hhead) rather than from pass B partials
+  int32_t n_tc_segs, n_tc_ctas, max_tc_segs;
+  cake::TcSegment* h_tc_segs;     // pinned
+  int32_t* h_tc_index;            // pinned: cta_seg [n_sm+1] then pair_seg [max_pairs+1]
+  cake::TcSegment* d_tc_segs;
+  int32_t* d_tc_cta_seg;
+  int32_t* d_tc_pair_seg;
+  float4* d_tc_rowpart;           // [max_tc_segs][128]
+  float* d_lse2_tc;               // [max_requests][H_kv][128], rows in tile order i*G + h
+  double* d_hhead;                // [max_requests][H_q] entropy per query head from pass A
 };
 
 namespace cake {
@@ -98,6 +119,10 @@ void count_launch(int64_t n = 1);
 // score_simt.cu
 int32_t launch_score_simt(cake_ctx* ctx, const void* q_win, const void* k, const float* lse,
                           cudaStream_t st);
+// score_tc.cu
+bool tc_path_supported(const cake_config& c);
+int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const float* lse,
+                        cudaStream_t st);
 // cascade.cu
 int32_t launch_finalize_layer(cake_ctx* ctx, int32_t layer, cudaStream_t st);
 int32_t launch_pool(cake_ctx* ctx, cudaStream_t st);

@@ -49,6 +49,46 @@ __global__ void finalize_layer(const float* __restrict__ colpart, const ReqInfo*
   }
 }
 
+// Same for the tensor-core path: partials are indexed by segment, and the entropy of
+// each query head may already have been reduced from the row pass (hhead).
+__global__ void finalize_layer_tc(const float* __restrict__ colpart,
+                                  const int32_t* __restrict__ pair_seg,
+                                  const double* __restrict__ hhead, int use_hhead,
+                                  double* __restrict__ dH, double* __restrict__ dV,
+                                  double* __restrict__ dP, int32_t* __restrict__ status, int layer,
+                                  int L, int Hq, int Hkv, double inv_tau1, double inv_tau2) {
+  __shared__ double sh[2][256];
+  const int req = blockIdx.x;
+  const int G = Hq / Hkv;
+  double hsum = 0.0, vsum = 0.0;
+  for (int h = threadIdx.x; h < Hq; h += blockDim.x) {
+    const int g = h / G, hl = h - g * G;
+    const int pair = req * Hkv + g;
+    double a = 0.0, b = 0.0;
+    for (int sg = pair_seg[pair]; sg < pair_seg[pair + 1]; ++sg) {
+      const float* p = colpart + ((size_t)sg * G + hl) * 2;
+      a += (double)p[0];
+      b += (double)p[1];
+    }
+    hsum += use_hhead ? hhead[(size_t)req * Hq + h] : -0.6931471805599453 * a;
+    vsum += b;
+  }
+  sh[0][threadIdx.x] = hsum;
+  sh[1][threadIdx.x] = vsum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double H = 0.0, V = 0.0;
+    for (int t = 0; t < blockDim.x; ++t) { H += sh[0][t]; V += sh[1][t]; }
+    H /= (double)Hq;
+    V /= (double)Hq;
+    const double P = pow(H, inv_tau1) * pow(V, inv_tau2);
+    dH[(size_t)req * L + layer] = H;
+    dV[(size_t)req * L + layer] = V;
+    dP[(size_t)req * L + layer] = P;
+    if (!(P >= 0.0) || isinf(P)) raise_status(status, CAKE_ERR_NONFINITE);
+  }
+}
+
 // --------------------------------------------------------------------- pool
 // fresh[g][t] = pool(raw[g][.]) over the request's non-window tokens; window
 // slots get +inf (Section 4.3).
@@ -397,6 +437,14 @@ evict_layers(const float* __restrict__ fresh, float* __restrict__ list_vals,
 int32_t launch_finalize_layer(cake_ctx* ctx, int32_t layer, cudaStream_t st) {
   const cake_config& c = ctx->cfg;
   if (ctx->n_req == 0) return CAKE_OK;
+  if (ctx->use_tc) {
+    finalize_layer_tc<<<ctx->n_req, 128, 0, st>>>(
+        ctx->d_colpart, ctx->d_tc_pair_seg, ctx->d_hhead, ctx->hhead_from_rows ? 1 : 0, ctx->d_H,
+        ctx->d_V, ctx->d_P, ctx->d_status, layer, c.n_layers, c.n_q_heads, c.n_kv_heads,
+        1.0 / (double)c.tau1, 1.0 / (double)c.tau2);
+    count_launch();
+    return cuda_status(cudaGetLastError());
+  }
   finalize_layer<<<ctx->n_req, 128, 0, st>>>(ctx->d_colpart, ctx->d_req, ctx->d_H, ctx->d_V,
                                               ctx->d_P, ctx->d_status, layer, c.n_layers,
                                               c.n_q_heads, c.n_kv_heads, 1.0 / (double)c.tau1,

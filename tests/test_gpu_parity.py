@@ -402,3 +402,36 @@ def test_generator_is_bit_identical_on_cpu_and_gpu():
     q0, k0, v0 = synth.layer_inputs(w, 1, "cpu")
     q1, k1, v1 = synth.layer_inputs(w, 1, "cuda")
     assert torch.equal(q0, q1.cpu()) and torch.equal(k0, k1.cpu()) and torch.equal(v0, v1.cpu())
+
+
+def test_simt_and_tensor_core_paths_agree_on_bf16(monkeypatch):
+    """bf16 inputs normally take the tcgen05 kernels; the SIMT kernels must give
+    the same indicators and preferences (both within tolerance of the oracle)."""
+    w = SMALL_CASES["gqa-bf16"]()
+    qs, ks, vs = harness.device_inputs(w)
+    ref = oracle_scores(w, qs, ks)
+    res = {}
+    for path in ("tc", "simt"):
+        monkeypatch.setenv("CAKE_SCORE_PATH", path)
+        cake = harness.cake_for(w)
+        assert cake.uses_tensor_cores() == (path == "tc")
+        cake.begin(w.cu_seqlens)
+        inds = []
+        for l in range(w.n_layers):
+            cake.score_layer(l, qs[l], ks[l])
+            inds.append(cake.get_indicators(l).cpu().numpy())
+            cake.allocate(l)
+            cake.evict(l)
+        H, V, P = (x.cpu().numpy() for x in cake.get_preferences())
+        assert cake.status() == 0
+        res[path] = (inds, H, V, P)
+        cake.destroy()
+    n = w.seq_lens[0] - w.window
+    for path in res:
+        inds, H, V, P = res[path]
+        for l in range(w.n_layers):
+            assert_close(inds[l][:, :n], ref[l][0]["indicator"], f"{path} indicator l{l}")
+            assert_close(H[0, l], ref[l][0]["H"], f"{path} H")
+            assert_close(V[0, l], ref[l][0]["V"], f"{path} V")
+    for l in range(w.n_layers):
+        assert_close(res["tc"][0][l][:, :n], res["simt"][0][l][:, :n], "tc vs simt", rtol=1e-4)
