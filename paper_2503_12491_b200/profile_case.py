@@ -1,0 +1,60 @@
+"""A reduced case of the eviction path, sized for profiler captures.
+
+    python -m paper_2503_12491_b200.profile_case [--workload 4] [--layers 2] [--steps 1]
+
+Runs the first `--layers` layers of a benchmark workload (same shapes per layer,
+budget scaled with the layer count) through begin / score / allocate / evict /
+compact.  Every layer's K is still larger than the L2 cache at workloads 4 and 5,
+so DRAM counters stay meaningful, while only a few GB are held on the device and
+a capture that replays each kernel many times ends by itself.  Prints the time
+of the last step; that figure is for orientation only, never a benchmark value.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import harness, synth
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", type=int, default=4)
+    ap.add_argument("--layers", type=int, default=2)
+    ap.add_argument("--steps", type=int, default=1)
+    ap.add_argument("--warmup", type=int, default=1)
+    args = ap.parse_args()
+
+    full = synth.workload(args.workload)
+    L = max(1, min(args.layers, full.n_layers))
+    w = synth.scaled(full, n_layers=L, total_budget=full.total_budget // full.n_layers * L)
+    torch.cuda.set_device(0)
+    qs, ks, vs = harness.device_inputs(w)
+    cake = harness.cake_for(w)
+    cake.begin(w.cu_seqlens)
+    rows = cake.packed_rows_bound()
+    bufs = dict(k_out=torch.empty(rows, w.head_dim, dtype=w.torch_dtype, device="cuda"),
+                v_out=torch.empty(rows, w.head_dim, dtype=w.torch_dtype, device="cuda"),
+                row_offsets=torch.empty(len(w.seq_lens) * L + 1, dtype=torch.int64, device="cuda"),
+                positions=torch.empty(rows, dtype=torch.int32, device="cuda"))
+    ms = None
+    for it in range(args.warmup + args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        cake.run(qs, ks, vs, w.cu_seqlens, **bufs)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+    status = cake.status()
+    print(json.dumps({"workload": w.name, "layers": L, "tokens": w.total_tokens,
+                      "last_step_ms": ms, "device_status": status,
+                      "retained_rows": int(bufs["row_offsets"][-1])}))
+    cake.destroy()
+    if status != 0:
+        raise SystemExit(1)
+
+
+if __name__ == "__main__":
+    main()
