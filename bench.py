@@ -267,10 +267,10 @@ def main():
     out_bytes = 2 * retained_rows * w.head_dim * esize
     ideal = k_bytes + q_bytes + out_bytes
 
-    # dominant kernel: the window-score pass with the larger share of the step;
+    # dominant kernel: the window-score kernel (both passes in one launch);
     # algorithmic bytes per launch = one layer's K read once + its window Q
     phase_ms = {k: v["ms"] / args.steps for k, v in prof.items()}
-    dom = max(("score_rows", "score_cols"), key=lambda k: prof[k]["ms"])
+    dom = "score"
     dom_ms = prof[dom]["ms"] / max(prof[dom]["spans"], 1)
     per_launch_bytes = (k_bytes + q_bytes) / L
     achieved = per_launch_bytes / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else None

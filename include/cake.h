@@ -168,13 +168,12 @@ int32_t cake_set_preferences(cake_ctx* ctx, int32_t n_layers_set, const double* 
 int32_t cake_status(cake_ctx* ctx, int32_t* device_status_out, void* stream);
 
 /* ---- tracing ------------------------------------------------------------ */
-#define CAKE_PROF_SCORE_ROWS  0  /* window scores, pass A: row max / sum (softmax denominators) */
-#define CAKE_PROF_SCORE_COLS  1  /* window scores, pass B: column statistics -> raw indicator   */
-#define CAKE_PROF_FINALIZE    2  /* preference + pooling                                         */
-#define CAKE_PROF_ALLOCATE    3
-#define CAKE_PROF_EVICT       4
-#define CAKE_PROF_COMPACT     5
-#define CAKE_PROF_KINDS       6
+#define CAKE_PROF_SCORE       0  /* window scores: softmax denominators and column statistics   */
+#define CAKE_PROF_FINALIZE    1  /* preference + pooling                                         */
+#define CAKE_PROF_ALLOCATE    2
+#define CAKE_PROF_EVICT       3
+#define CAKE_PROF_COMPACT     4
+#define CAKE_PROF_KINDS       5
 /* While enabled, every stage of the path brackets its kernels with CUDA events
  * on the caller's stream (this perturbs back-to-back launches slightly). */
 int32_t cake_profile_enable(cake_ctx* ctx, int32_t on);

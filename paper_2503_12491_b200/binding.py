@@ -30,7 +30,7 @@ EXPORTS = [
     "cake_set_preferences", "cake_status", "cake_strerror", "cake_launch_count",
     "cake_profile_enable", "cake_profile_read", "cake_uses_tensor_cores",
 ]
-PROF_KINDS = ["score_rows", "score_cols", "finalize", "allocate", "evict", "compact"]
+PROF_KINDS = ["score", "finalize", "allocate", "evict", "compact"]
 
 
 class CakeConfig(ctypes.Structure):

@@ -62,9 +62,9 @@ void free_ctx(cake_ctx* c) {
   cudaFree(c->d_budget[0]); cudaFree(c->d_budget[1]); cudaFree(c->d_status); cudaFree(c->d_raw);
   cudaFree(c->d_fresh); cudaFree(c->list_vals); cudaFree(c->list_pos); cudaFree(c->d_lse2);
   cudaFree(c->d_rowpart); cudaFree(c->d_colpart);
-  cudaFree(c->d_tc_segs); cudaFree(c->d_tc_cta_seg); cudaFree(c->d_tc_pair_seg);
+  cudaFree(c->d_tc_ops); cudaFree(c->d_tc_index); cudaFree(c->d_tc_sync);
   cudaFree(c->d_tc_rowpart); cudaFree(c->d_lse2_tc); cudaFree(c->d_hhead);
-  if (c->h_tc_segs) cudaFreeHost(c->h_tc_segs);
+  if (c->h_tc_ops) cudaFreeHost(c->h_tc_ops);
   if (c->h_tc_index) cudaFreeHost(c->h_tc_index);
   if (c->h_req) cudaFreeHost(c->h_req);
   if (c->h_units) cudaFreeHost(c->h_units);
@@ -148,19 +148,25 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
     x->use_tc = tc_path_supported(c) && !(force && strcmp(force, "simt") == 0);
   }
   const int64_t max_pairs = R * c.n_kv_heads;
-  x->max_tc_segs = (int32_t)(max_pairs + x->n_sm + 1);
+  x->max_pairs = (int32_t)max_pairs;
   {
-    const size_t a = (size_t)x->max_units * c.n_kv_heads, b = (size_t)x->max_tc_segs;
+    const int64_t segs = tc_max_segments(c, x->n_sm);
+    if (x->use_tc && segs > ((int64_t)1 << 24)) { free_ctx(x); return CAKE_ERR_ARG; }
+    x->max_tc_segs = (int32_t)segs;
+    x->max_tc_ops = (int32_t)(3 * segs + 8);
+  }
+  {
+    const size_t a = (size_t)x->max_units * c.n_kv_heads, b = (size_t)x->max_tc_segs * kScoreGroups;
     ok = ok && dev_alloc(&x->d_colpart, (a > b ? a : b) * G * 2) == cudaSuccess;
   }
   if (x->use_tc) {
-    ok = ok && cudaMallocHost((void**)&x->h_tc_segs, sizeof(TcSegment) * x->max_tc_segs) == cudaSuccess;
-    ok = ok && cudaMallocHost((void**)&x->h_tc_index,
-                              sizeof(int32_t) * (x->n_sm + 1 + max_pairs + 1)) == cudaSuccess;
-    ok = ok && dev_alloc(&x->d_tc_segs, x->max_tc_segs) == cudaSuccess;
-    ok = ok && dev_alloc(&x->d_tc_cta_seg, x->n_sm + 1) == cudaSuccess;
-    ok = ok && dev_alloc(&x->d_tc_pair_seg, max_pairs + 1) == cudaSuccess;
-    ok = ok && dev_alloc(&x->d_tc_rowpart, (size_t)x->max_tc_segs * 128) == cudaSuccess;
+    const size_t n_index = 2 * (size_t)(max_pairs + 1) + 2 * (size_t)(x->n_sm + 1);
+    ok = ok && cudaMallocHost((void**)&x->h_tc_ops, sizeof(ScoreOp) * x->max_tc_ops) == cudaSuccess;
+    ok = ok && cudaMallocHost((void**)&x->h_tc_index, sizeof(int32_t) * n_index) == cudaSuccess;
+    ok = ok && dev_alloc(&x->d_tc_ops, x->max_tc_ops) == cudaSuccess;
+    ok = ok && dev_alloc(&x->d_tc_index, n_index) == cudaSuccess;
+    ok = ok && dev_alloc(&x->d_tc_sync, 2 * (size_t)max_pairs) == cudaSuccess;
+    ok = ok && dev_alloc(&x->d_tc_rowpart, (size_t)x->max_tc_segs * kScoreGroups * 128) == cudaSuccess;
     ok = ok && dev_alloc(&x->d_lse2_tc, (size_t)max_pairs * 128) == cudaSuccess;
     ok = ok && dev_alloc(&x->d_hhead, (size_t)R * c.n_q_heads) == cudaSuccess;
   }
@@ -225,41 +231,8 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
     }
     if (list_off > ctx->list_elems || nu > ctx->max_units) return CAKE_ERR_CAPACITY;
     if (ctx->use_tc) {
-      // Flatten (request, KV head, 128-key tile) and give every CTA an equal contiguous share;
-      // a share is cut into segments where it crosses a (request, KV head) boundary.
-      const int TILE = 128;
-      int64_t W = 0;
-      for (int r = 0; r < n_req; ++r) W += (int64_t)c.n_kv_heads * ((ctx->h_req[r].N + TILE - 1) / TILE);
-      const int n_cta = (int)(W < ctx->n_sm ? W : ctx->n_sm);
-      int32_t* cta_seg = ctx->h_tc_index;
-      int32_t* pair_seg = ctx->h_tc_index + ctx->n_sm + 1;
-      int ns = 0, cta = 0;
-      int64_t flat = 0;                                    // tiles before the current pair
-      cta_seg[0] = 0;
-      for (int r = 0; r < n_req; ++r) {
-        const int tiles = (ctx->h_req[r].N + TILE - 1) / TILE;
-        for (int g = 0; g < c.n_kv_heads; ++g) {
-          pair_seg[r * c.n_kv_heads + g] = ns;
-          int t0 = 0;
-          while (t0 < tiles) {
-            // the CTA owning flat tile (flat + t0); its share ends at ceil-split boundary
-            while ((int64_t)(cta + 1) * W / n_cta <= flat + t0) cta_seg[++cta] = ns;
-            const int64_t share_end = (int64_t)(cta + 1) * W / n_cta;
-            const int t1 = (int)((share_end - flat) < tiles ? (share_end - flat) : tiles);
-            TcSegment& sgm = ctx->h_tc_segs[ns++];
-            sgm.req = r; sgm.g = g; sgm.key0 = t0 * TILE;
-            const int kend = t1 * TILE < ctx->h_req[r].N ? t1 * TILE : ctx->h_req[r].N;
-            sgm.nkeys = kend - t0 * TILE;
-            t0 = t1;
-          }
-          flat += tiles;
-        }
-      }
-      while (cta < n_cta) cta_seg[++cta] = ns;
-      pair_seg[n_req * c.n_kv_heads] = ns;
-      if (ns > ctx->max_tc_segs) return CAKE_ERR_CAPACITY;
-      ctx->n_tc_segs = ns;
-      ctx->n_tc_ctas = n_cta;
+      const int32_t prc = tc_build_plan(ctx, n_req);
+      if (prc != CAKE_OK) return prc;
     }
     ctx->n_units = nu;
     ctx->packed_rows_bound = bound;
@@ -268,19 +241,22 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
                                   cudaMemcpyHostToDevice, st));
     CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_units, ctx->h_units, sizeof(ScoreUnit) * nu,
                                   cudaMemcpyHostToDevice, st));
-    if (ctx->use_tc) {
-      CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_tc_segs, ctx->h_tc_segs, sizeof(TcSegment) * ctx->n_tc_segs,
+    if (ctx->use_tc && ctx->n_tc_ctas > 0) {
+      const size_t n_index = 2 * (size_t)(n_req * c.n_kv_heads + 1) + 2 * (size_t)(ctx->n_sm + 1);
+      CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_tc_ops, ctx->h_tc_ops,
+                                    sizeof(ScoreOp) * (ctx->n_tc_ops_full + ctx->n_tc_ops_b),
                                     cudaMemcpyHostToDevice, st));
-      CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_tc_cta_seg, ctx->h_tc_index,
-                                    sizeof(int32_t) * (ctx->n_tc_ctas + 1), cudaMemcpyHostToDevice, st));
-      CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_tc_pair_seg, ctx->h_tc_index + ctx->n_sm + 1,
-                                    sizeof(int32_t) * (n_req * c.n_kv_heads + 1),
+      CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_tc_index, ctx->h_tc_index, sizeof(int32_t) * n_index,
                                     cudaMemcpyHostToDevice, st));
     }
     CAKE_CUDA_TRY(cudaEventRecord(ctx->upload_done, st));
     ctx->upload_pending = true;
   }
-  if (n_req == 0) { ctx->n_units = 0; ctx->packed_rows_bound = 0; ctx->n_tc_segs = 0; ctx->n_tc_ctas = 0; }
+  if (n_req == 0) { ctx->n_units = 0; ctx->packed_rows_bound = 0; ctx->n_tc_ctas = 0; }
+  if (ctx->use_tc) {
+    ctx->tc_epoch = 0;
+    CAKE_CUDA_TRY(cudaMemsetAsync(ctx->d_tc_sync, 0, sizeof(uint32_t) * 2 * ctx->max_pairs, st));
+  }
   ctx->n_req = n_req;
   ctx->total_tokens = T;
   ctx->n_ind = ctx->n_pref = ctx->n_evicted = 0;

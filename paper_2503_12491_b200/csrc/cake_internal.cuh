@@ -12,6 +12,7 @@ namespace cake {
 constexpr int kMaxRows = 128;        // G * S_w rows handled per KV head
 constexpr int kSimtTileKeys = 64;    // keys per tile of the SIMT score kernels
 constexpr int kSimtThreads = 256;
+constexpr int kScoreGroups = 3;      // statistics warp groups per CTA of the tensor-core score kernel
 
 // One request of the current batch (device copy in ctx->d_req).
 struct ReqInfo {
@@ -33,13 +34,17 @@ struct ScoreUnit {
   int32_t pad;
 };
 
-// A run of consecutive keys of one (request, KV head) handled by one CTA of the
-// tensor-core score kernels.
-struct TcSegment {
+// One step of a CTA's program in the tensor-core score kernel: a run of consecutive
+// keys of one (request, KV head) in pass A (phase 0, row statistics) or pass B (phase 1,
+// column statistics).  `seg` numbers the partial results the step writes (one per
+// statistics warp group).
+struct ScoreOp {
   int32_t req;
   int32_t g;
   int32_t key0;
   int32_t nkeys;
+  int32_t phase;
+  int32_t seg;
 };
 
 struct LayerPtrs {
@@ -101,13 +106,19 @@ struct cake_ctx {
   // ---- tensor-core score path ----
   bool use_tc;
   bool hhead_from_rows;    // entropy came from pass A (d_hhead) rather than from pass B partials
-  int32_t n_tc_segs, n_tc_ctas, max_tc_segs;
-  cake::TcSegment* h_tc_segs;     // pinned
-  int32_t* h_tc_index;            // pinned: cta_seg [n_sm+1] then pair_seg [max_pairs+1]
-  cake::TcSegment* d_tc_segs;
-  int32_t* d_tc_cta_seg;
-  int32_t* d_tc_pair_seg;
-  float4* d_tc_rowpart;           // [max_tc_segs][128]
+  int32_t n_tc_ctas, max_tc_segs, max_pairs;
+  int32_t n_tc_asegs, n_tc_bsegs;          // pass-A / pass-B segments per layer
+  int32_t n_tc_ops_full, n_tc_ops_b, max_tc_ops;
+  uint32_t tc_epoch;              // both-pass launches since cake_begin
+  cake::ScoreOp* h_tc_ops;        // pinned: [both-pass programs][pass-B-only programs]
+  cake::ScoreOp* d_tc_ops;
+  // pinned / device index block of the current batch, P = n_req * H_kv pairs:
+  //   pair_aseg [P+1] | pair_bseg [P+1] | cta_op of the both-pass programs [n_sm+1]
+  //   | cta_op of the pass-B-only programs [n_sm+1]
+  int32_t* h_tc_index;
+  int32_t* d_tc_index;
+  uint32_t* d_tc_sync;            // [max_pairs] delivered partial rows, then [max_pairs] flags
+  float4* d_tc_rowpart;           // [max_tc_segs][kScoreGroups][128]
   float* d_lse2_tc;               // [max_requests][H_kv][128], rows in tile order i*G + h
   double* d_hhead;                // [max_requests][H_q] entropy per query head from pass A
 };
@@ -121,6 +132,8 @@ int32_t launch_score_simt(cake_ctx* ctx, const void* q_win, const void* k, const
                           cudaStream_t st);
 // score_tc.cu
 bool tc_path_supported(const cake_config& c);
+int64_t tc_max_segments(const cake_config& c, int n_sm);
+int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req);
 int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const float* lse,
                         cudaStream_t st);
 // cascade.cu

@@ -49,8 +49,9 @@ __global__ void finalize_layer(const float* __restrict__ colpart, const ReqInfo*
   }
 }
 
-// Same for the tensor-core path: partials are indexed by segment, and the entropy of
-// each query head may already have been reduced from the row pass (hhead).
+// Same for the tensor-core path: partials are indexed by (pass-B segment, statistics
+// group), and the entropy of each query head may already have been reduced from the
+// row pass (hhead).
 __global__ void finalize_layer_tc(const float* __restrict__ colpart,
                                   const int32_t* __restrict__ pair_seg,
                                   const double* __restrict__ hhead, int use_hhead,
@@ -65,7 +66,7 @@ __global__ void finalize_layer_tc(const float* __restrict__ colpart,
     const int g = h / G, hl = h - g * G;
     const int pair = req * Hkv + g;
     double a = 0.0, b = 0.0;
-    for (int sg = pair_seg[pair]; sg < pair_seg[pair + 1]; ++sg) {
+    for (int sg = pair_seg[pair] * kScoreGroups; sg < pair_seg[pair + 1] * kScoreGroups; ++sg) {
       const float* p = colpart + ((size_t)sg * G + hl) * 2;
       a += (double)p[0];
       b += (double)p[1];
@@ -439,7 +440,7 @@ int32_t launch_finalize_layer(cake_ctx* ctx, int32_t layer, cudaStream_t st) {
   if (ctx->n_req == 0) return CAKE_OK;
   if (ctx->use_tc) {
     finalize_layer_tc<<<ctx->n_req, 128, 0, st>>>(
-        ctx->d_colpart, ctx->d_tc_pair_seg, ctx->d_hhead, ctx->hhead_from_rows ? 1 : 0, ctx->d_H,
+        ctx->d_colpart, ctx->d_tc_index + (ctx->n_req * c.n_kv_heads + 1), ctx->d_hhead, ctx->hhead_from_rows ? 1 : 0, ctx->d_H,
         ctx->d_V, ctx->d_P, ctx->d_status, layer, c.n_layers, c.n_q_heads, c.n_kv_heads,
         1.0 / (double)c.tau1, 1.0 / (double)c.tau2);
     count_launch();

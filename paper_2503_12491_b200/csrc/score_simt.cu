@@ -335,7 +335,7 @@ int32_t run(cake_ctx* ctx, const void* q_win, const void* k, const float* lse, c
   }
   const dim3 grid(ctx->n_units, c.n_kv_heads);
   const int64_t n_lse = (int64_t)ctx->n_req * c.n_q_heads * c.window;
-  int sp = prof_begin(ctx, CAKE_PROF_SCORE_ROWS, st);
+  int sp = prof_begin(ctx, CAKE_PROF_SCORE, st);
   if (lse) {
     lse_to_base2<<<(unsigned)((n_lse + 255) / 256), 256, 0, st>>>(lse, ctx->d_lse2, n_lse);
     count_launch();
@@ -348,7 +348,7 @@ int32_t run(cake_ctx* ctx, const void* q_win, const void* k, const float* lse, c
     count_launch(2);
   }
   prof_end(ctx, sp, st);
-  sp = prof_begin(ctx, CAKE_PROF_SCORE_COLS, st);
+  sp = prof_begin(ctx, CAKE_PROF_SCORE, st);
   score_colstats_simt<T><<<grid, NT, smem, st>>>(
       (const T*)q_win, (const T*)k, ctx->d_req, ctx->d_units, ctx->d_lse2, ctx->d_raw,
       ctx->d_colpart, c.n_q_heads, c.n_kv_heads, c.window, c.head_dim, ctx->total_tokens, scale2,

@@ -1,26 +1,39 @@
-// Window-score kernels for bf16 inputs on the sm_100a tensor cores.
+// Window-score kernel for bf16 inputs on the sm_100a tensor cores: one persistent
+// launch per layer runs both passes over the keys.
 //
-// Both passes stream K tiles of 128 keys through shared memory with TMA
-// (no multicast), multiply them against the resident window queries with
-// tcgen05.mma (bf16 operands, fp32 accumulators in tensor memory) and reduce
-// the accumulator tile on chip; the S_w x N score matrix never reaches HBM.
-//
-//   pass A (rows)   D[row][key]  = Q K^T : one thread owns one window row and
-//                   keeps its running max / sum (softmax denominator, Eq. 2) and
+//   pass A (rows)   D[row][key]  = Q K^T : one thread owns one window row and keeps
+//                   its running max / sum (softmax denominator, Eq. 2) and
 //                   sum e*log2(e) (row entropy, Eq. 4).
 //   pass B (cols)   D[key][row]  = K Q^T : one thread owns one key and reduces its
 //                   normalised column over the window rows: group-mean attention,
 //                   Mean + gamma Var (Eq. 11) and the per-head Var (Eq. 5).
 //
-// Warp roles in a CTA of 320 threads: warp 0 issues TMA loads, warp 1 owns the
-// tensor-memory allocation and issues the MMAs, warps 2..9 are two groups of
-// four "statistics" warps that take alternate accumulator tiles.  Every wait on
-// an mbarrier is bounded; a timed-out wait raises CAKE_ERR_TIMEOUT and the CTA
+// K tiles of 128 keys stream through shared memory with TMA (no multicast), are
+// multiplied against the resident window queries with tcgen05.mma (bf16 operands,
+// fp32 accumulators in tensor memory) and reduced on chip; the S_w x N score matrix
+// never reaches HBM.
+//
+// Schedule.  The (request, KV head) pairs of a layer are grouped into waves of at
+// most kWaveBytes of K.  Every CTA owns the same slice of a wave in both passes and runs
+//     A(wave 0), A(wave 1), B(wave 0), A(wave 2), B(wave 1), ... , B(last wave)
+// so pass B re-reads a wave's K from L2 shortly after pass A brought it in, and DRAM
+// sees K once.  Pass B of a pair needs the pair's softmax denominators, i.e. every
+// CTA's pass-A partial rows: whoever delivers the last partial merges them all and
+// publishes a per-pair flag; the pass A of the next wave sits between a pair's pass A
+// and its pass B, so the wait on that flag is normally already satisfied.
+//
+// Warp roles in a CTA of 512 threads: warp 0 issues TMA loads, warp 1 owns the
+// tensor-memory allocation and issues the MMAs, warps 4..15 are three independent
+// groups of four "statistics" warps that take accumulator tiles round-robin; a group
+// synchronises only with itself and writes its own partial results.  Every wait
+// (mbarrier or flag) is bounded; a timed-out wait raises CAKE_ERR_TIMEOUT and the CTA
 // drains and exits.
 #include "cake_internal.cuh"
 
 #include <cuda.h>
 #include <math_constants.h>
+
+#include <vector>
 
 namespace cake {
 namespace {
@@ -28,22 +41,31 @@ namespace {
 constexpr int TILE = 128;            // keys per tile
 constexpr int STAGES = 4;            // K tiles in flight
 constexpr int NBUF = 4;              // accumulator buffers (4 x 128 of the 512 TMEM columns)
-constexpr int TC_THREADS = 320;
+constexpr int NWG = kScoreGroups;    // statistics warp groups
+constexpr int STAT_THREADS = NWG * 128;
+constexpr int TC_THREADS = 128 + STAT_THREADS;
 constexpr int SLAB_BYTES = TILE * 128;   // one 64-element slab of a 128-row tile
 constexpr long long kSpinLimit = 4000000000ll;   // cycles (~2 s) before a wait gives up
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLazyMax = 8.f;      // pass A rescales only when the row max grows by 2^8
+constexpr int64_t kWaveBytes = 32ll << 20;
 
 struct TcParams {
-  const TcSegment* segs;
-  const int32_t* cta_seg;       // [n_cta + 1]
+  const ScoreOp* ops;
+  const int32_t* cta_op;        // [n_cta + 1]
   const ReqInfo* reqs;
-  float* lse2;                  // [req][H_kv][128] in tile row order r' = i*G + h
-  float4* rowpart;              // pass A out: [segment][128] (m, z_all, z_win, w)
+  const int32_t* pair_aseg;     // [pairs + 1] pass-A segment ranges per pair
+  uint32_t* pair_cnt;           // [pairs] delivered pass-A partials (monotonic over layers)
+  uint32_t* pair_flag;          // [pairs] epoch of the last published denominators (or null)
+  float* lse2;                  // [pair][128] in tile row order r' = i*G + h
+  float4* rowpart;              // pass A out: [A-segment][group][128] (m, z_all, z_win, w)
   float* raw;                   // pass B out: [H_kv][T]
-  float* colpart;               // pass B out: [segment][G][2]
+  float* colpart;               // pass B out: [B-segment][group][G][2]
+  double* hhead;                // [req][H_q] entropy per query head
   int32_t* status;
   int64_t T;
-  int Hkv, G, Sw, rows, d;
+  uint32_t epoch;
+  int Hkv, Hq, Sw, rows, d;
   float scale2, gamma, bessel;
 };
 
@@ -158,63 +180,89 @@ __device__ __forceinline__ uint32_t instr_desc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(uint32_t* p, uint32_t v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
 struct Smem {
-  uint8_t* q;          // 2 slabs x 128 rows x 128 B
+  uint8_t* q;          // 2 buffers x (2 slabs x 128 rows x 128 B)
   uint8_t* k;          // STAGES x (2 slabs x 128 rows x 128 B)
   uint64_t* full;      // [STAGES]
   uint64_t* empty;     // [STAGES]
   uint64_t* acc_full;  // [NBUF]
   uint64_t* acc_empty; // [NBUF]
-  uint64_t* q_full;
-  uint64_t* q_empty;
+  uint64_t* q_full;    // [2]
+  uint64_t* q_empty;   // [2]
   uint32_t* tmem_holder;
-  float* lse;          // [128]
-  float* xchg;         // [128 * 4]
+  uint32_t* last_flag; // [NWG]
+  float* lse;          // [NWG][128]  per group: denominators (pass B) / row exchange (merge)
+  float* red;          // [NWG][4 warps][16]
 };
 
-constexpr size_t kSmemBytes = 1024 /*align*/ + 2 * SLAB_BYTES + (size_t)STAGES * 2 * SLAB_BYTES + 256 +
-                              128 * 4 + 128 * 16 + 64;
+constexpr size_t kQBytes = 2 * SLAB_BYTES;
+constexpr size_t kSmemBytes = 1024 /*align*/ + 2 * kQBytes + (size_t)STAGES * 2 * SLAB_BYTES + 256 +
+                              NWG * 128 * 4 + NWG * 64 * 4 + 64;
 
 __device__ __forceinline__ Smem carve(uint8_t* base) {
   Smem s;
   uint8_t* p = (uint8_t*)(((uintptr_t)base + 1023) & ~(uintptr_t)1023);
-  s.q = p;                    p += 2 * SLAB_BYTES;
+  s.q = p;                    p += 2 * kQBytes;
   s.k = p;                    p += (size_t)STAGES * 2 * SLAB_BYTES;
   s.full = (uint64_t*)p;      p += 8 * STAGES;
   s.empty = (uint64_t*)p;     p += 8 * STAGES;
   s.acc_full = (uint64_t*)p;  p += 8 * NBUF;
   s.acc_empty = (uint64_t*)p; p += 8 * NBUF;
-  s.q_full = (uint64_t*)p;    p += 8;
-  s.q_empty = (uint64_t*)p;   p += 8;
+  s.q_full = (uint64_t*)p;    p += 16;
+  s.q_empty = (uint64_t*)p;   p += 16;
   s.tmem_holder = (uint32_t*)p; p += 16;
+  s.last_flag = (uint32_t*)p;   p += 16;
   p = (uint8_t*)(((uintptr_t)p + 15) & ~(uintptr_t)15);
-  s.lse = (float*)p;          p += 128 * 4;
-  s.xchg = (float*)p;
+  s.lse = (float*)p;          p += NWG * 128 * 4;
+  s.red = (float*)p;
   return s;
 }
 
+// Merge of two partial softmax rows (m, z_all, z_win, w) with base-2 exponents;
+// w = sum over observed keys of e * (logit2 - m).
+__device__ __forceinline__ float4 merge_rows(float4 a, float4 b) {
+  if (b.x == -CUDART_INF_F) return a;
+  if (a.x == -CUDART_INF_F) return b;
+  const float mn = fmaxf(a.x, b.x);
+  const float fa = exp2f(a.x - mn), fb = exp2f(b.x - mn);
+  float4 o;
+  o.x = mn;
+  o.y = a.y * fa + b.y * fb;
+  o.z = a.z * fa + b.z * fb;
+  o.w = fa * fmaf(a.x - mn, a.y - a.z, a.w) + fb * fmaf(b.x - mn, b.y - b.z, b.w);
+  return o;
+}
+
 // ------------------------------------------------------------------ kernel
-template <bool kCols, bool kEntropy>
+template <int G, bool kEntropyB>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
-                const TcParams P) {
+score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
+                   const TcParams P) {
   extern __shared__ uint8_t smem_raw[];
   const Smem S = carve(smem_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_slab = P.d / 64;
   const uint32_t stage_bytes = (uint32_t)(TILE * P.d * 2);
   const int rows_pad = (P.rows + 15) & ~15;
-  const int seg_lo = P.cta_seg[blockIdx.x], seg_hi = P.cta_seg[blockIdx.x + 1];
+  const int op_lo = P.cta_op[blockIdx.x], op_hi = P.cta_op[blockIdx.x + 1];
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], 1); }
     for (int i = 0; i < NBUF; ++i) { mbar_init(&S.acc_full[i], 1); mbar_init(&S.acc_empty[i], 128); }
-    mbar_init(S.q_full, 1);
-    mbar_init(S.q_empty, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&S.q_full[i], 1); mbar_init(&S.q_empty[i], 1); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // rows of the query tile that TMA never writes must read as zero
-  for (int i = threadIdx.x; i < 2 * SLAB_BYTES / 16; i += TC_THREADS)
+  // rows of the query tiles that TMA never writes must read as zero
+  for (int i = threadIdx.x; i < (int)(2 * kQBytes / 16); i += TC_THREADS)
     reinterpret_cast<uint4*>(S.q)[i] = make_uint4(0, 0, 0, 0);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (warp == 1) {
@@ -236,20 +284,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
       uint32_t t = 0, qn = 0;
       bool ok = true;
-      for (int sg = seg_lo; sg < seg_hi && ok; ++sg) {
-        const TcSegment seg = P.segs[sg];
-        const ReqInfo rq = P.reqs[seg.req];
-        const int nkeys = kCols ? min(seg.nkeys, rq.n - seg.key0) : seg.nkeys;
-        if (nkeys <= 0) continue;
-        // previous segment's MMAs must be done with the query tile
-        ok = mbar_wait(S.q_empty, (qn & 1) ^ 1, P.status);
+      for (int oi = op_lo; oi < op_hi && ok; ++oi) {
+        const ScoreOp op = P.ops[oi];
+        if (op.nkeys <= 0) continue;
+        const ReqInfo rq = P.reqs[op.req];
+        const int qb = qn & 1;
+        // the MMAs of the op that used this query buffer two ops ago must be done
+        ok = mbar_wait(&S.q_empty[qb], ((qn >> 1) & 1) ^ 1, P.status);
         ++qn;
         if (!ok) break;
-        mbar_expect_tx(S.q_full, (uint32_t)(P.rows * P.d * 2));
+        mbar_expect_tx(&S.q_full[qb], (uint32_t)(P.rows * P.d * 2));
         for (int sl = 0; sl < n_slab; ++sl)
-          tma_load_4d(S.q + sl * SLAB_BYTES, &q_map, S.q_full, sl * 64, seg.g * P.G, 0, seg.req);
-        const int64_t row0 = (int64_t)seg.g * P.T + rq.cu + seg.key0;
-        const int ntiles = (nkeys + TILE - 1) / TILE;
+          tma_load_4d(S.q + qb * kQBytes + sl * SLAB_BYTES, &q_map, &S.q_full[qb], sl * 64, op.g * G,
+                      0, op.req);
+        const int64_t row0 = (int64_t)op.g * P.T + rq.cu + op.key0;
+        const int ntiles = (op.nkeys + TILE - 1) / TILE;
         for (int it = 0; it < ntiles; ++it, ++t) {
           const int s = t % STAGES;
           ok = mbar_wait(&S.empty[s], ((t / STAGES) & 1) ^ 1, P.status);
@@ -264,22 +313,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       const uint32_t issued = t;
       for (uint32_t u = issued > STAGES ? issued - STAGES : 0; u < issued; ++u)
         mbar_wait(&S.full[u % STAGES], (u / STAGES) & 1, P.status);
+      for (uint32_t u = qn > 2 ? qn - 2 : 0; u < qn; ++u)
+        mbar_wait(&S.q_full[u & 1], (u >> 1) & 1, P.status);
     }
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = kCols ? instr_desc(128, rows_pad) : instr_desc(128, TILE);
       uint32_t t = 0, qn = 0;
       bool ok = true;
-      for (int sg = seg_lo; sg < seg_hi && ok; ++sg) {
-        const TcSegment seg = P.segs[sg];
-        const ReqInfo rq = P.reqs[seg.req];
-        const int nkeys = kCols ? min(seg.nkeys, rq.n - seg.key0) : seg.nkeys;
-        if (nkeys <= 0) continue;
-        ok = mbar_wait(S.q_full, qn & 1, P.status);
+      for (int oi = op_lo; oi < op_hi && ok; ++oi) {
+        const ScoreOp op = P.ops[oi];
+        if (op.nkeys <= 0) continue;
+        const uint32_t idesc = op.phase ? instr_desc(128, rows_pad) : instr_desc(128, TILE);
+        const int qb = qn & 1;
+        ok = mbar_wait(&S.q_full[qb], (qn >> 1) & 1, P.status);
         ++qn;
         if (!ok) break;
-        const int ntiles = (nkeys + TILE - 1) / TILE;
+        const uint32_t qaddr = smem_u32(S.q + qb * kQBytes);
+        const int ntiles = (op.nkeys + TILE - 1) / TILE;
         for (int it = 0; it < ntiles; ++it, ++t) {
           const int s = t % STAGES, b = t % NBUF;
           ok = mbar_wait(&S.acc_empty[b], ((t / NBUF) & 1) ^ 1, P.status);
@@ -288,194 +339,186 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           if (!ok) break;
           tc_fence_after();
           const uint32_t kaddr = smem_u32(S.k + (size_t)s * 2 * SLAB_BYTES);
-          const uint32_t qaddr = smem_u32(S.q);
           const uint32_t tmem_d = tmem_base + (uint32_t)(b * 128);
           for (int sl = 0; sl < n_slab; ++sl) {
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
               const uint64_t kd = smem_desc(kaddr + sl * SLAB_BYTES + ks * 32);
               const uint64_t qd = smem_desc(qaddr + sl * SLAB_BYTES + ks * 32);
-              if (kCols) umma_bf16(tmem_d, kd, qd, idesc, (sl | ks) != 0);
-              else       umma_bf16(tmem_d, qd, kd, idesc, (sl | ks) != 0);
+              if (op.phase) umma_bf16(tmem_d, kd, qd, idesc, (sl | ks) != 0);
+              else          umma_bf16(tmem_d, qd, kd, idesc, (sl | ks) != 0);
             }
           }
           umma_commit(&S.empty[s]);
           umma_commit(&S.acc_full[b]);
         }
-        umma_commit(S.q_empty);        // query tile free once every MMA of the segment has run
+        umma_commit(&S.q_empty[qb]);     // query buffer free once every MMA of the op has run
       }
     }
-  } else {
+  } else if (warp >= 4) {
     // ------------------------------------------------ statistics warps
-    const int wg = (warp - 2) >> 2;                 // 0 or 1: takes tiles of matching parity
+    const int wg = (warp - 4) >> 2;                 // 0..NWG-1: takes tiles t with t % NWG == wg
     const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
     const int lane_row = quad * 32 + lane;          // accumulator lane (row in pass A, key in pass B)
-    const int sthread = threadIdx.x - 64;           // 0..255 among the statistics threads
+    const int bar_wg = 1 + wg;                      // named barrier of this warp group
+    float* lse_wg = S.lse + wg * 128;
+    float* red_wg = S.red + wg * 64;
     uint32_t t = 0;
     bool ok = true;
-    for (int sg = seg_lo; sg < seg_hi; ++sg) {
-      const TcSegment seg = P.segs[sg];
-      const ReqInfo rq = P.reqs[seg.req];
-      const int nkeys = kCols ? min(seg.nkeys, rq.n - seg.key0) : seg.nkeys;
-      const int ntiles = nkeys > 0 ? (nkeys + TILE - 1) / TILE : 0;
-      if (kCols) {
+    for (int oi = op_lo; oi < op_hi; ++oi) {
+      const ScoreOp op = P.ops[oi];
+      if (op.nkeys <= 0) continue;
+      const ReqInfo rq = P.reqs[op.req];
+      const int ntiles = (op.nkeys + TILE - 1) / TILE;
+      const int pair = op.req * P.Hkv + op.g;
+      if (op.phase) {
         // ---------------- pass B: thread = key, columns = rows r' = i*G + h
-        named_bar(1, 256);                          // previous segment done with S.lse / S.xchg
-        if (sthread < 128)
-          S.lse[sthread] = sthread < P.rows
-              ? P.lse2[((size_t)seg.req * P.Hkv + seg.g) * 128 + sthread] : 0.f;
-        named_bar(1, 256);
-        float vacc[8], hs[8];
+        if (lane_row == 0 && P.pair_flag) {         // denominators of this pair published?
+          const long long t0 = clock64();
+          while (ld_acquire(&P.pair_flag[pair]) != P.epoch) {
+            if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); break; }
+            __nanosleep(32);
+          }
+        }
+        named_bar(bar_wg, 128);
+        lse_wg[lane_row] = lane_row < P.rows ? __ldcg(&P.lse2[(size_t)pair * 128 + lane_row]) : 0.f;
+        named_bar(bar_wg, 128);
+        float vacc[G], hs[G];
 #pragma unroll
-        for (int h = 0; h < 8; ++h) { vacc[h] = 0.f; hs[h] = 0.f; }
-        const float inv_sw = 1.f / (float)P.Sw, inv_g = 1.f / (float)P.G;
+        for (int h = 0; h < G; ++h) { vacc[h] = 0.f; hs[h] = 0.f; }
+        const float inv_sw = 1.f / (float)P.Sw, inv_g = 1.f / (float)G;
         for (int it = 0; it < ntiles; ++it, ++t) {
-          if ((int)(t & 1) != wg) continue;
+          if ((int)(t % NWG) != wg) continue;
           const int b = t % NBUF;
           if (ok) ok = mbar_wait(&S.acc_full[b], (t / NBUF) & 1, P.status);
           if (!ok) continue;
           tc_fence_after();
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * 128);
-          float s1[8], s2[8], a1 = 0.f, a2 = 0.f, hkeep[8];
+          float s1[G], s2[G], hk[G], a2 = 0.f;
 #pragma unroll
-          for (int h = 0; h < 8; ++h) { s1[h] = 0.f; s2[h] = 0.f; hkeep[h] = hs[h]; }
+          for (int h = 0; h < G; ++h) { s1[h] = 0.f; s2[h] = 0.f; hk[h] = 0.f; }
           for (int c0 = 0; c0 < P.rows; c0 += 32) {
             float v[32];
             tmem_ld32(taddr + c0, v);
             // 32 columns = 32/G window rows x G heads
-            if (P.G == 4) {
 #pragma unroll
-              for (int ii = 0; ii < 8; ++ii) {
-                const float4 l4 = *reinterpret_cast<const float4*>(&S.lse[c0 + ii * 4]);
-                const float t0 = fmaf(v[ii * 4 + 0], P.scale2, -l4.x);
-                const float t1 = fmaf(v[ii * 4 + 1], P.scale2, -l4.y);
-                const float t2 = fmaf(v[ii * 4 + 2], P.scale2, -l4.z);
-                const float t3 = fmaf(v[ii * 4 + 3], P.scale2, -l4.w);
-                const float p0 = ex2(t0), p1 = ex2(t1), p2 = ex2(t2), p3 = ex2(t3);
-                if (kEntropy) {
-                  hs[0] = fmaf(p0, t0, hs[0]); hs[1] = fmaf(p1, t1, hs[1]);
-                  hs[2] = fmaf(p2, t2, hs[2]); hs[3] = fmaf(p3, t3, hs[3]);
-                }
-                s1[0] += p0; s2[0] = fmaf(p0, p0, s2[0]);
-                s1[1] += p1; s2[1] = fmaf(p1, p1, s2[1]);
-                s1[2] += p2; s2[2] = fmaf(p2, p2, s2[2]);
-                s1[3] += p3; s2[3] = fmaf(p3, p3, s2[3]);
-                const float a = ((p0 + p1) + (p2 + p3)) * inv_g;
-                a1 += a; a2 = fmaf(a, a, a2);
-              }
-            } else {
-              // generic group size (1, 2 or 8): column c = i*G + h
-              for (int e = 0; e < 32; e += P.G) {
-                float a = 0.f;
-                for (int h = 0; h < P.G; ++h) {
-                  const float tt = fmaf(v[e + h], P.scale2, -S.lse[c0 + e + h]);
-                  const float p = ex2(tt);
+            for (int ii = 0; ii < 32 / G; ++ii) {
+              float a = 0.f;
 #pragma unroll
-                  for (int hh = 0; hh < 8; ++hh)
-                    if (hh == h) {
-                      s1[hh] += p; s2[hh] = fmaf(p, p, s2[hh]);
-                      if (kEntropy) hs[hh] = fmaf(p, tt, hs[hh]);
-                    }
-                  a += p;
-                }
-                a *= inv_g;
-                a1 += a; a2 = fmaf(a, a, a2);
+              for (int h = 0; h < G; ++h) {
+                const float tt = fmaf(v[ii * G + h], P.scale2, -lse_wg[c0 + ii * G + h]);
+                const float p = ex2(tt);
+                s1[h] += p;
+                s2[h] = fmaf(p, p, s2[h]);
+                if (kEntropyB) hk[h] = fmaf(p, tt, hk[h]);
+                a += p;
               }
+              a2 = fmaf(a, a, a2);
             }
           }
           tc_fence_before();
           mbar_arrive(&S.acc_empty[b]);
-          const int j = seg.key0 + it * TILE + lane_row;          // key index inside the request
-          if (j < rq.n && it * TILE + lane_row < nkeys) {
-            const float mean = a1 * inv_sw;
-            const float var = fmaxf(a2 * inv_sw - mean * mean, 0.f) * P.bessel;
-            P.raw[(size_t)seg.g * P.T + rq.cu + j] = fmaf(P.gamma, var, mean);
+          const int j = op.key0 + it * TILE + lane_row;          // key index inside the request
+          if (j < rq.n && it * TILE + lane_row < op.nkeys) {
+            float a1 = 0.f;
 #pragma unroll
-            for (int h = 0; h < 8; ++h) {
+            for (int h = 0; h < G; ++h) {
+              a1 += s1[h];
               const float mh = s1[h] * inv_sw;
               vacc[h] += fmaxf(s2[h] * inv_sw - mh * mh, 0.f) * P.bessel;
+              if (kEntropyB) hs[h] += hk[h];
             }
-          } else {
-#pragma unroll
-            for (int h = 0; h < 8; ++h) hs[h] = hkeep[h];      // key outside the observed range
+            const float mean = a1 * inv_g * inv_sw;
+            const float var = fmaxf(a2 * inv_g * inv_g * inv_sw - mean * mean, 0.f) * P.bessel;
+            P.raw[(size_t)op.g * P.T + rq.cu + j] = fmaf(P.gamma, var, mean);
           }
         }
-        // fixed-order reduction of vacc over the 256 statistics threads
-        named_bar(1, 256);
+        // fixed-order reduction over the group's threads
 #pragma unroll
-        for (int h = 0; h < 8; ++h) {
+        for (int h = 0; h < G; ++h) {
           float x = vacc[h], y = hs[h];
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) {
             x += __shfl_xor_sync(0xffffffffu, x, o);
             y += __shfl_xor_sync(0xffffffffu, y, o);
           }
-          if (lane == 0) { S.xchg[(warp - 2) * 16 + h] = x; S.xchg[(warp - 2) * 16 + 8 + h] = y; }
+          if (lane == 0) { red_wg[quad * 16 + h] = x; red_wg[quad * 16 + 8 + h] = y; }
         }
-        named_bar(1, 256);
-        if (sthread < P.G) {
+        named_bar(bar_wg, 128);
+        if (lane_row < G) {
           float acc = 0.f, hacc = 0.f;
-          for (int w2 = 0; w2 < 8; ++w2) {
-            acc += S.xchg[w2 * 16 + sthread];
-            hacc += S.xchg[w2 * 16 + 8 + sthread];
+#pragma unroll
+          for (int w2 = 0; w2 < 4; ++w2) {
+            acc += red_wg[w2 * 16 + lane_row];
+            hacc += red_wg[w2 * 16 + 8 + lane_row];
           }
-          P.colpart[((size_t)sg * P.G + sthread) * 2 + 0] = hacc;
-          P.colpart[((size_t)sg * P.G + sthread) * 2 + 1] = acc;
+          float* dst = P.colpart + (((size_t)op.seg * NWG + wg) * G + lane_row) * 2;
+          dst[0] = hacc;
+          dst[1] = acc;
         }
       } else {
         // ---------------- pass A: thread = window row r' = i*G + h, columns = keys
-        const int i_row = lane_row / P.G;
+        const int i_row = lane_row / G;
         const int last = rq.n + i_row;                 // last key this row may attend to
         float m = -CUDART_INF_F, z = 0.f, zwin = 0.f, w = 0.f;
         for (int it = 0; it < ntiles; ++it, ++t) {
-          if ((int)(t & 1) != wg) continue;
+          if ((int)(t % NWG) != wg) continue;
           const int b = t % NBUF;
           if (ok) ok = mbar_wait(&S.acc_full[b], (t / NBUF) & 1, P.status);
           if (!ok) continue;
           tc_fence_after();
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * 128);
-          const int key0 = seg.key0 + it * TILE;
-          const bool interior = key0 + TILE <= rq.n && it * TILE + TILE <= nkeys;
+          const int key0 = op.key0 + it * TILE;
+          const bool interior = key0 + TILE <= rq.n && it * TILE + TILE <= op.nkeys;
 #pragma unroll 1
           for (int c0 = 0; c0 < TILE; c0 += 32) {
             float v[32];
             tmem_ld32(taddr + c0, v);
             if (interior) {
-              float cm = v[0];
+              float c4[4] = {v[0], v[1], v[2], v[3]};
 #pragma unroll
-              for (int e = 1; e < 32; ++e) cm = fmaxf(cm, v[e]);
-              const float mn = fmaxf(m, cm * P.scale2);
-              const float f = ex2(m - mn);                     // 0 on the first chunk
-              const float dm = (m == -CUDART_INF_F) ? 0.f : (m - mn);
-              w = f * fmaf(dm, z - zwin, w);
-              z *= f; zwin *= f;
-              m = mn;
+              for (int e = 4; e < 32; ++e) c4[e & 3] = fmaxf(c4[e & 3], v[e]);
+              const float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3])) * P.scale2;
+              if (cm > m + kLazyMax) {                        // rare after the first tiles
+                const float mn = cm;
+                const float f = ex2(m - mn);                  // 0 while m = -inf
+                const float dm = (m == -CUDART_INF_F) ? 0.f : (m - mn);
+                w = f * fmaf(dm, z - zwin, w);
+                z *= f; zwin *= f;
+                m = mn;
+              }
+              float zc[4] = {0.f, 0.f, 0.f, 0.f}, wc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
                 const float tt = fmaf(v[e], P.scale2, -m);
                 const float ee = ex2(tt);
-                z += ee;
-                w = fmaf(ee, tt, w);
+                zc[e & 3] += ee;
+                wc[e & 3] = fmaf(ee, tt, wc[e & 3]);
               }
+              z += (zc[0] + zc[1]) + (zc[2] + zc[3]);
+              w += (wc[0] + wc[1]) + (wc[2] + wc[3]);
             } else {
               float cm = -CUDART_INF_F;
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
                 const int j = key0 + c0 + e;
-                const bool vis = (it * TILE + c0 + e < nkeys) && j <= last;
+                const bool vis = (it * TILE + c0 + e < op.nkeys) && j <= last;
                 cm = vis ? fmaxf(cm, v[e]) : cm;
               }
               if (cm != -CUDART_INF_F) {
-                const float mn = fmaxf(m, cm * P.scale2);
-                const float f = ex2(m - mn);
-                const float dm = (m == -CUDART_INF_F) ? 0.f : (m - mn);
-                w = f * fmaf(dm, z - zwin, w);
-                z *= f; zwin *= f;
-                m = mn;
+                cm *= P.scale2;
+                if (cm > m) {
+                  const float mn = cm;
+                  const float f = ex2(m - mn);
+                  const float dm = (m == -CUDART_INF_F) ? 0.f : (m - mn);
+                  w = f * fmaf(dm, z - zwin, w);
+                  z *= f; zwin *= f;
+                  m = mn;
+                }
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                   const int j = key0 + c0 + e;
-                  const bool vis = (it * TILE + c0 + e < nkeys) && j <= last;
+                  const bool vis = (it * TILE + c0 + e < op.nkeys) && j <= last;
                   const bool obs = j < rq.n;
                   const float tt = fmaf(v[e], P.scale2, -m);
                   const float ee = vis ? ex2(tt) : 0.f;
@@ -489,27 +532,48 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           tc_fence_before();
           mbar_arrive(&S.acc_empty[b]);
         }
-        // merge the two groups' partial rows, group 0 writes
-        named_bar(1, 256);
-        if (wg == 1) {
-          reinterpret_cast<float4*>(S.xchg)[lane_row] = make_float4(m, z, zwin, w);
+        // deliver this group's partial rows of the segment
+        __stcg(&P.rowpart[((size_t)op.seg * NWG + wg) * 128 + lane_row], make_float4(m, z, zwin, w));
+        __threadfence();
+        named_bar(bar_wg, 128);
+        if (lane_row == 0) {
+          const uint32_t nseg = (uint32_t)(P.pair_aseg[pair + 1] - P.pair_aseg[pair]) * NWG;
+          const uint32_t old = atomicAdd(&P.pair_cnt[pair], 1u);
+          S.last_flag[wg] = (old + 1u == nseg * P.epoch) ? 1u : 0u;
         }
-        named_bar(1, 256);
-        if (wg == 0) {
-          const float4 o = reinterpret_cast<const float4*>(S.xchg)[lane_row];
-          float mn = fmaxf(m, o.x);
-          float4 outv = make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
-          if (mn != -CUDART_INF_F) {
-            const float fa = (m == -CUDART_INF_F) ? 0.f : ex2(m - mn);
-            const float fb = (o.x == -CUDART_INF_F) ? 0.f : ex2(o.x - mn);
-            const float da = (m == -CUDART_INF_F) ? 0.f : (m - mn);
-            const float db = (o.x == -CUDART_INF_F) ? 0.f : (o.x - mn);
-            outv.x = mn;
-            outv.y = z * fa + o.y * fb;
-            outv.z = zwin * fa + o.z * fb;
-            outv.w = fa * fmaf(da, z - zwin, w) + fb * fmaf(db, o.y - o.z, o.w);
+        named_bar(bar_wg, 128);
+        if (S.last_flag[wg]) {
+          // the pair's last partial: merge them all and publish the denominators
+          __threadfence();
+          const float4 none = make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
+          float4 part[4] = {none, none, none, none};
+          const int s_lo = P.pair_aseg[pair] * NWG, s_hi = P.pair_aseg[pair + 1] * NWG;
+          for (int sg = s_lo; sg < s_hi; sg += 8) {           // eight loads in flight per thread
+            float4 pv[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+              pv[u] = sg + u < s_hi ? __ldcg(&P.rowpart[(size_t)(sg + u) * 128 + lane_row]) : none;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) part[u & 3] = merge_rows(part[u & 3], pv[u]);
           }
-          P.rowpart[(size_t)sg * 128 + lane_row] = outv;
+          const float4 tot = merge_rows(merge_rows(part[0], part[1]), merge_rows(part[2], part[3]));
+          float hrow = 0.f;
+          if (lane_row < P.rows) {
+            const float lz = log2f(tot.y);
+            __stcg(&P.lse2[(size_t)pair * 128 + lane_row], tot.x + lz);
+            // sum_j p log2 p over the observed keys = (w - log2(z) * z_obs) / z
+            hrow = (tot.w - lz * (tot.y - tot.z)) / tot.y;
+          }
+          lse_wg[lane_row] = hrow;
+          named_bar(bar_wg, 128);
+          if (lane_row < G) {                        // head h = rows h, h+G, h+2G, ...
+            double acc2 = 0.0;
+            for (int i = lane_row; i < P.rows; i += G) acc2 += (double)lse_wg[i];
+            P.hhead[(size_t)op.req * P.Hq + op.g * G + lane_row] = -0.6931471805599453 * acc2;
+          }
+          __threadfence();
+          named_bar(bar_wg, 128);
+          if (lane_row == 0) st_release(&P.pair_flag[pair], P.epoch);
         }
       }
     }
@@ -521,45 +585,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512)
                  : "memory");
-  }
-}
-
-// Merge the row partials of every (request, KV head): lse2 per row and the
-// entropy per query head.  Rows are in tile order r' = i*G + h.
-__global__ void tc_rowstats_combine(const float4* __restrict__ rowpart,
-                                    const int32_t* __restrict__ pair_seg,
-                                    float* __restrict__ lse2, double* __restrict__ hhead, int Hkv,
-                                    int G, int rows, int Hq) {
-  __shared__ float hrow[128];
-  const int req = blockIdx.x, g = blockIdx.y, r = threadIdx.x;
-  const int pair = req * Hkv + g;
-  float m = -CUDART_INF_F, z = 0.f, zw = 0.f, w = 0.f;
-  for (int sg = pair_seg[pair]; sg < pair_seg[pair + 1]; ++sg) {
-    const float4 p = rowpart[(size_t)sg * 128 + r];
-    if (p.x == -CUDART_INF_F) continue;
-    const float mn = fmaxf(m, p.x);
-    const float fa = (m == -CUDART_INF_F) ? 0.f : exp2f(m - mn);
-    const float fb = exp2f(p.x - mn);
-    const float da = (m == -CUDART_INF_F) ? 0.f : (m - mn);
-    const float db = p.x - mn;
-    w = fa * fmaf(da, z - zw, w) + fb * fmaf(db, p.y - p.z, p.w);
-    z = z * fa + p.y * fb;
-    zw = zw * fa + p.z * fb;
-    m = mn;
-  }
-  float h = 0.f;
-  if (r < rows) {
-    const float lz = log2f(z);
-    lse2[(size_t)pair * 128 + r] = m + lz;
-    // sum_j p log2 p = (w - log2(z) * z_obs) / z
-    h = (w - lz * (z - zw)) / z;
-  }
-  hrow[r] = h;
-  __syncthreads();
-  if (r < G) {                                  // head h = rows r, r+G, r+2G, ...
-    double acc = 0.0;
-    for (int i = r; i < rows; i += G) acc += (double)hrow[i];
-    hhead[(size_t)req * Hq + g * G + r] = -0.6931471805599453 * acc;
   }
 }
 
@@ -592,6 +617,49 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+
+template <int G>
+cudaError_t launch_g(bool entropy_b, int n_cta, cudaStream_t st, const CUtensorMap& qmap,
+                     const CUtensorMap& kmap, const TcParams& P) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(score_fused_kernel<G, false>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(score_fused_kernel<G, true>,
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  if (entropy_b) score_fused_kernel<G, true><<<n_cta, TC_THREADS, kSmemBytes, st>>>(qmap, kmap, P);
+  else           score_fused_kernel<G, false><<<n_cta, TC_THREADS, kSmemBytes, st>>>(qmap, kmap, P);
+  return cudaGetLastError();
+}
+
+// Cuts the `tiles` tiles of one (request, head) pair, which start at flat tile index `flat`
+// of a wave of `W` tiles shared by `n_cta` CTAs (slot c owns flat tiles
+// [c*W/n_cta, (c+1)*W/n_cta)), into per-slot segments; slot c belongs to CTA (c+rot)%n_cta.
+void cut_pair(std::vector<std::vector<ScoreOp>>& per_cta, int rot, int n_cta, int64_t W, int64_t flat,
+              int tiles, int keys, int req, int g, int phase, int32_t& seg_counter) {
+  int t0 = 0;
+  while (t0 < tiles) {
+    const int64_t f = flat + t0;
+    int c = (int)(f * n_cta / W);
+    while (c + 1 < n_cta && (int64_t)(c + 1) * W / n_cta <= f) ++c;
+    while (c > 0 && (int64_t)c * W / n_cta > f) --c;
+    const int64_t share_end = (int64_t)(c + 1) * W / n_cta;
+    const int t1 = (int)((share_end - flat) < tiles ? (share_end - flat) : tiles);
+    ScoreOp op;
+    op.req = req; op.g = g; op.key0 = t0 * TILE;
+    const int kend = t1 * TILE < keys ? t1 * TILE : keys;
+    op.nkeys = kend - t0 * TILE;
+    op.phase = phase;
+    op.seg = seg_counter++;
+    per_cta[(c + rot) % n_cta].push_back(op);
+    t0 = t1;
+  }
+}
+
 }  // namespace
 
 bool tc_path_supported(const cake_config& c) {
@@ -601,10 +669,105 @@ bool tc_path_supported(const cake_config& c) {
          rows <= 128 && (G == 1 || G == 2 || G == 4 || G == 8) && c.window <= 256;
 }
 
+// Upper bound on the segments of one pass: every pair gives one segment plus one per CTA
+// boundary inside its wave; two consecutive waves hold more than kWaveBytes of K, and there
+// are no more waves than pairs.
+int64_t tc_max_segments(const cake_config& c, int n_sm) {
+  const int64_t pairs = (int64_t)c.max_requests * c.n_kv_heads;
+  const int64_t bytes = (int64_t)c.n_kv_heads * c.max_total_tokens * c.head_dim * 2;
+  int64_t waves = 2 * (bytes / kWaveBytes) + 2;
+  if (waves > pairs) waves = pairs;
+  return pairs + waves * n_sm;
+}
+
+// Builds the per-CTA programs of the batch in ctx->h_req[0..n_req): `full` = both passes
+// interleaved by wave, `bonly` = pass B alone (denominators supplied by the caller).
+int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
+  const cake_config& c = ctx->cfg;
+  const int Hkv = c.n_kv_heads;
+  const int n_pairs = n_req * Hkv;
+  int64_t tilesA_total = 0;
+  for (int r = 0; r < n_req; ++r) tilesA_total += (int64_t)Hkv * ((ctx->h_req[r].N + TILE - 1) / TILE);
+  const int n_cta = (int)(tilesA_total < ctx->n_sm ? tilesA_total : ctx->n_sm);
+  ctx->n_tc_ctas = n_cta;
+  ctx->n_tc_ops_full = ctx->n_tc_ops_b = 0;
+  ctx->n_tc_asegs = ctx->n_tc_bsegs = 0;
+  if (n_cta == 0) return CAKE_OK;
+
+  std::vector<int> wave_begin{0};                          // waves of consecutive pairs
+  {
+    int64_t bytes = 0;
+    for (int p = 0; p < n_pairs; ++p) {
+      const int64_t pb = (int64_t)ctx->h_req[p / Hkv].N * c.head_dim * 2;
+      if (bytes > 0 && bytes + pb > kWaveBytes) { wave_begin.push_back(p); bytes = 0; }
+      bytes += pb;
+    }
+    wave_begin.push_back(n_pairs);
+  }
+  const int n_waves = (int)wave_begin.size() - 1;
+  std::vector<std::vector<ScoreOp>> full(n_cta), bonly(n_cta), wa(n_cta), wb(n_cta), wb_prev(n_cta);
+  int32_t aseg = 0, bseg = 0;
+  int32_t* pair_aseg = ctx->h_tc_index;                    // [pairs+1]
+  int32_t* pair_bseg = ctx->h_tc_index + (n_pairs + 1);    // [pairs+1]
+  int rot = 0;
+  for (int wv = 0; wv < n_waves; ++wv) {
+    int64_t WA = 0;
+    for (int p = wave_begin[wv]; p < wave_begin[wv + 1]; ++p)
+      WA += (ctx->h_req[p / Hkv].N + TILE - 1) / TILE;
+    for (int cta = 0; cta < n_cta; ++cta) { wa[cta].clear(); wb[cta].clear(); }
+    int64_t fa = 0;
+    for (int p = wave_begin[wv]; p < wave_begin[wv + 1]; ++p) {
+      const int r = p / Hkv, g = p % Hkv;
+      const ReqInfo& rq = ctx->h_req[r];
+      const int ta = (rq.N + TILE - 1) / TILE, tb = (rq.n + TILE - 1) / TILE;
+      pair_aseg[p] = aseg;
+      pair_bseg[p] = bseg;
+      cut_pair(wa, rot, n_cta, WA, fa, ta, rq.N, r, g, 0, aseg);
+      // pass B walks the same flat tile positions, so a CTA re-reads the tiles it brought in
+      if (tb > 0) cut_pair(wb, rot, n_cta, WA, fa, tb, rq.n, r, g, 1, bseg);
+      fa += ta;
+    }
+    rot = (rot + 37) % n_cta;             // a wave's remainder tiles land on different CTAs each time
+    for (int cta = 0; cta < n_cta; ++cta) {
+      full[cta].insert(full[cta].end(), wa[cta].begin(), wa[cta].end());
+      if (wv > 0) full[cta].insert(full[cta].end(), wb_prev[cta].begin(), wb_prev[cta].end());
+      bonly[cta].insert(bonly[cta].end(), wb[cta].begin(), wb[cta].end());
+    }
+    wb_prev.swap(wb);
+  }
+  for (int cta = 0; cta < n_cta; ++cta)
+    full[cta].insert(full[cta].end(), wb_prev[cta].begin(), wb_prev[cta].end());
+  pair_aseg[n_pairs] = aseg;
+  pair_bseg[n_pairs] = bseg;
+  if (aseg > ctx->max_tc_segs || bseg > ctx->max_tc_segs) return CAKE_ERR_CAPACITY;
+
+  int32_t* cta_full = ctx->h_tc_index + 2 * (n_pairs + 1);   // [n_sm+1]
+  int32_t* cta_b = cta_full + (ctx->n_sm + 1);               // [n_sm+1]
+  int64_t total = 0;
+  for (int cta = 0; cta < n_cta; ++cta) total += (int64_t)(full[cta].size() + bonly[cta].size());
+  if (total > ctx->max_tc_ops) return CAKE_ERR_CAPACITY;
+  int32_t o = 0;
+  for (int cta = 0; cta < n_cta; ++cta) {
+    cta_full[cta] = o;
+    for (const ScoreOp& op : full[cta]) ctx->h_tc_ops[o++] = op;
+  }
+  cta_full[n_cta] = o;
+  ctx->n_tc_ops_full = o;
+  for (int cta = 0; cta < n_cta; ++cta) {
+    cta_b[cta] = o;
+    for (const ScoreOp& op : bonly[cta]) ctx->h_tc_ops[o++] = op;
+  }
+  cta_b[n_cta] = o;
+  ctx->n_tc_ops_b = o - ctx->n_tc_ops_full;
+  ctx->n_tc_asegs = aseg;
+  ctx->n_tc_bsegs = bseg;
+  return CAKE_OK;
+}
+
 int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const float* lse,
                         cudaStream_t st) {
   const cake_config& c = ctx->cfg;
-  if (ctx->n_tc_segs == 0) return CAKE_OK;
+  if (ctx->n_tc_ctas == 0) return CAKE_OK;
   if ((int64_t)c.n_kv_heads * ctx->total_tokens >= ((int64_t)1 << 31)) return CAKE_ERR_ARG;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return CAKE_ERR_CUDA;
@@ -633,52 +796,52 @@ int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const f
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return CAKE_ERR_CUDA;
   }
-  static bool attr_done = false;
-  if (!attr_done) {
-    CAKE_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<false, false>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-    CAKE_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<true, false>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-    CAKE_CUDA_TRY(cudaFuncSetAttribute(score_tc_kernel<true, true>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-    attr_done = true;
-  }
+  const int n_pairs = ctx->n_req * c.n_kv_heads;
   TcParams P;
-  P.segs = ctx->d_tc_segs;
-  P.cta_seg = ctx->d_tc_cta_seg;
+  P.ops = ctx->d_tc_ops;
   P.reqs = ctx->d_req;
+  P.pair_aseg = ctx->d_tc_index;
+  P.pair_cnt = ctx->d_tc_sync;
   P.lse2 = ctx->d_lse2_tc;
   P.rowpart = ctx->d_tc_rowpart;
   P.raw = ctx->d_raw;
   P.colpart = ctx->d_colpart;
+  P.hhead = ctx->d_hhead;
   P.status = ctx->d_status;
   P.T = ctx->total_tokens;
-  P.Hkv = c.n_kv_heads; P.G = G; P.Sw = c.window; P.rows = ctx->rows; P.d = c.head_dim;
+  P.Hkv = c.n_kv_heads; P.Hq = c.n_q_heads; P.Sw = c.window; P.rows = ctx->rows; P.d = c.head_dim;
   P.scale2 = kLog2e / sqrtf((float)c.head_dim);
   P.gamma = c.gamma;
   P.bessel = c.var_ddof ? (float)c.window / (float)(c.window - 1) : 1.f;
 
-  const dim3 pairs(ctx->n_req, c.n_kv_heads);
-  int sp = prof_begin(ctx, CAKE_PROF_SCORE_ROWS, st);
+  const int sp = prof_begin(ctx, CAKE_PROF_SCORE, st);
+  const int32_t* cta_full = ctx->d_tc_index + 2 * (n_pairs + 1);
   if (lse) {
+    // denominators supplied: pass B alone, entropy from its columns
+    const dim3 pairs(ctx->n_req, c.n_kv_heads);
     tc_lse_permute<<<pairs, 128, 0, st>>>(lse, ctx->d_lse2_tc, c.n_kv_heads, G, c.window);
-    CAKE_CUDA_TRY(cudaMemsetAsync(ctx->d_hhead, 0, sizeof(double) * ctx->n_req * c.n_q_heads, st));
     count_launch();
     ctx->hhead_from_rows = false;
+    P.cta_op = cta_full + (ctx->n_sm + 1);
+    P.pair_flag = nullptr;
+    P.epoch = 0;
   } else {
-    score_tc_kernel<false, false><<<ctx->n_tc_ctas, TC_THREADS, kSmemBytes, st>>>(qmap, kmap, P);
-    tc_rowstats_combine<<<pairs, 128, 0, st>>>(ctx->d_tc_rowpart, ctx->d_tc_pair_seg, ctx->d_lse2_tc,
-                                               ctx->d_hhead, c.n_kv_heads, G, ctx->rows, c.n_q_heads);
-    count_launch(2);
     ctx->hhead_from_rows = true;
+    P.cta_op = cta_full;
+    P.pair_flag = ctx->d_tc_sync + ctx->max_pairs;
+    P.epoch = ++ctx->tc_epoch;
   }
-  prof_end(ctx, sp, st);
-  sp = prof_begin(ctx, CAKE_PROF_SCORE_COLS, st);
-  if (lse) score_tc_kernel<true, true><<<ctx->n_tc_ctas, TC_THREADS, kSmemBytes, st>>>(qmap, kmap, P);
-  else     score_tc_kernel<true, false><<<ctx->n_tc_ctas, TC_THREADS, kSmemBytes, st>>>(qmap, kmap, P);
+  cudaError_t e;
+  const bool eb = lse != nullptr;
+  switch (G) {
+    case 1: e = launch_g<1>(eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
+    case 2: e = launch_g<2>(eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
+    case 4: e = launch_g<4>(eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
+    default: e = launch_g<8>(eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
+  }
   count_launch();
   prof_end(ctx, sp, st);
-  return cuda_status(cudaGetLastError());
+  return cuda_status(e);
 }
 
 }  // namespace cake
