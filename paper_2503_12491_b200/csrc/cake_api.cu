@@ -63,7 +63,7 @@ void free_ctx(cake_ctx* c) {
   cudaFree(c->d_fresh); cudaFree(c->list_vals); cudaFree(c->list_pos); cudaFree(c->d_lse2);
   cudaFree(c->d_rowpart); cudaFree(c->d_colpart);
   cudaFree(c->d_tc_ops); cudaFree(c->d_tc_index); cudaFree(c->d_tc_sync);
-  cudaFree(c->d_tc_rowpart); cudaFree(c->d_lse2_tc); cudaFree(c->d_hhead);
+  cudaFree(c->d_tc_rowpart); cudaFree(c->d_lse2_tc); cudaFree(c->d_hrow);
   if (c->h_tc_ops) cudaFreeHost(c->h_tc_ops);
   if (c->h_tc_index) cudaFreeHost(c->h_tc_index);
   if (c->h_req) cudaFreeHost(c->h_req);
@@ -168,7 +168,7 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
     ok = ok && dev_alloc(&x->d_tc_sync, 2 * (size_t)max_pairs) == cudaSuccess;
     ok = ok && dev_alloc(&x->d_tc_rowpart, (size_t)x->max_tc_segs * kScoreGroups * 128) == cudaSuccess;
     ok = ok && dev_alloc(&x->d_lse2_tc, (size_t)max_pairs * 128) == cudaSuccess;
-    ok = ok && dev_alloc(&x->d_hhead, (size_t)R * c.n_q_heads) == cudaSuccess;
+    ok = ok && dev_alloc(&x->d_hrow, (size_t)max_pairs * 128) == cudaSuccess;
   }
   ok = ok && cudaMemset(x->d_status, 0, sizeof(int32_t)) == cudaSuccess;
   ok = ok && cudaMemset(x->d_budget[0], 0, sizeof(int32_t) * R * c.n_layers) == cudaSuccess;

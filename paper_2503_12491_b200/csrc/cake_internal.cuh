@@ -105,7 +105,7 @@ struct cake_ctx {
   float* d_colpart;        // [max_units][H_kv][G][2] partial (sum p*log2 p, sum var) of phase B
   // ---- tensor-core score path ----
   bool use_tc;
-  bool hhead_from_rows;    // entropy came from pass A (d_hhead) rather than from pass B partials
+  bool hhead_from_rows;    // entropy came from pass A (d_hrow) rather than from pass B partials
   int32_t n_tc_ctas, max_tc_segs, max_pairs;
   int32_t n_tc_asegs, n_tc_bsegs;          // pass-A / pass-B segments per layer
   int32_t n_tc_ops_full, n_tc_ops_b, max_tc_ops;
@@ -117,10 +117,10 @@ struct cake_ctx {
   //   | cta_op of the pass-B-only programs [n_sm+1]
   int32_t* h_tc_index;
   int32_t* d_tc_index;
-  uint32_t* d_tc_sync;            // [max_pairs] delivered partial rows, then [max_pairs] flags
+  uint32_t* d_tc_sync;            // [max_pairs] delivered partial rows, then [max_pairs] merged rows
   float4* d_tc_rowpart;           // [max_tc_segs][kScoreGroups][128]
   float* d_lse2_tc;               // [max_requests][H_kv][128], rows in tile order i*G + h
-  double* d_hhead;                // [max_requests][H_q] entropy per query head from pass A
+  float* d_hrow;                  // [max_pairs][128] sum_j p log2 p per window row from pass A
 };
 
 namespace cake {

@@ -49,37 +49,49 @@ __global__ void finalize_layer(const float* __restrict__ colpart, const ReqInfo*
   }
 }
 
-// Same for the tensor-core path: partials are indexed by (pass-B segment, statistics
-// group), and the entropy of each query head may already have been reduced from the
-// row pass (hhead).
+// Same for the tensor-core path: one warp per query head.  Variance partials are indexed
+// by (pass-B segment, statistics group); the entropy comes either from the row pass
+// (hrow: sum_j p log2 p of every window row, tile row order r' = i*G + h) or, when the
+// caller supplied the denominators, from the column pass partials.
+__device__ inline double warp_sum_f64(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
 __global__ void finalize_layer_tc(const float* __restrict__ colpart,
                                   const int32_t* __restrict__ pair_seg,
-                                  const double* __restrict__ hhead, int use_hhead,
+                                  const float* __restrict__ hrow, int use_hrow, int rows,
                                   double* __restrict__ dH, double* __restrict__ dV,
                                   double* __restrict__ dP, int32_t* __restrict__ status, int layer,
                                   int L, int Hq, int Hkv, double inv_tau1, double inv_tau2) {
-  __shared__ double sh[2][256];
+  __shared__ double sh[2][32];
   const int req = blockIdx.x;
   const int G = Hq / Hkv;
-  double hsum = 0.0, vsum = 0.0;
-  for (int h = threadIdx.x; h < Hq; h += blockDim.x) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
+  double hsum = 0.0, vsum = 0.0;                         // per warp, over its heads
+  for (int h = warp; h < Hq; h += nwarp) {
     const int g = h / G, hl = h - g * G;
     const int pair = req * Hkv + g;
     double a = 0.0, b = 0.0;
-    for (int sg = pair_seg[pair] * kScoreGroups; sg < pair_seg[pair + 1] * kScoreGroups; ++sg) {
-      const float* p = colpart + ((size_t)sg * G + hl) * 2;
-      a += (double)p[0];
-      b += (double)p[1];
+    const int s_lo = pair_seg[pair] * kScoreGroups, s_hi = pair_seg[pair + 1] * kScoreGroups;
+    for (int sg = s_lo + lane; sg < s_hi; sg += 32) {
+      const float2 p = *reinterpret_cast<const float2*>(colpart + ((size_t)sg * G + hl) * 2);
+      a += (double)p.x;
+      b += (double)p.y;
     }
-    hsum += use_hhead ? hhead[(size_t)req * Hq + h] : -0.6931471805599453 * a;
-    vsum += b;
+    if (use_hrow) {
+      a = 0.0;
+      for (int r = hl + lane * G; r < rows; r += 32 * G) a += (double)hrow[(size_t)pair * 128 + r];
+    }
+    hsum += -0.6931471805599453 * warp_sum_f64(a);
+    vsum += warp_sum_f64(b);
   }
-  sh[0][threadIdx.x] = hsum;
-  sh[1][threadIdx.x] = vsum;
+  if (lane == 0) { sh[0][warp] = hsum; sh[1][warp] = vsum; }
   __syncthreads();
   if (threadIdx.x == 0) {
     double H = 0.0, V = 0.0;
-    for (int t = 0; t < blockDim.x; ++t) { H += sh[0][t]; V += sh[1][t]; }
+    for (int t = 0; t < nwarp; ++t) { H += sh[0][t]; V += sh[1][t]; }
     H /= (double)Hq;
     V /= (double)Hq;
     const double P = pow(H, inv_tau1) * pow(V, inv_tau2);
@@ -439,8 +451,9 @@ int32_t launch_finalize_layer(cake_ctx* ctx, int32_t layer, cudaStream_t st) {
   const cake_config& c = ctx->cfg;
   if (ctx->n_req == 0) return CAKE_OK;
   if (ctx->use_tc) {
-    finalize_layer_tc<<<ctx->n_req, 128, 0, st>>>(
-        ctx->d_colpart, ctx->d_tc_index + (ctx->n_req * c.n_kv_heads + 1), ctx->d_hhead, ctx->hhead_from_rows ? 1 : 0, ctx->d_H,
+    finalize_layer_tc<<<ctx->n_req, 1024, 0, st>>>(
+        ctx->d_colpart, ctx->d_tc_index + (ctx->n_req * c.n_kv_heads + 1), ctx->d_hrow,
+        ctx->hhead_from_rows ? 1 : 0, ctx->rows, ctx->d_H,
         ctx->d_V, ctx->d_P, ctx->d_status, layer, c.n_layers, c.n_q_heads, c.n_kv_heads,
         1.0 / (double)c.tau1, 1.0 / (double)c.tau2);
     count_launch();

@@ -18,12 +18,14 @@
 //     A(wave 0), A(wave 1), B(wave 0), A(wave 2), B(wave 1), ... , B(last wave)
 // so pass B re-reads a wave's K from L2 shortly after pass A brought it in, and DRAM
 // sees K once.  Pass B of a pair needs the pair's softmax denominators, i.e. every
-// CTA's pass-A partial rows: whoever delivers the last partial merges them all and
-// publishes a per-pair flag; the pass A of the next wave sits between a pair's pass A
-// and its pass B, so the wait on that flag is normally already satisfied.
+// CTA's pass-A partial rows.  The merge is spread over the grid by rows: one spare warp
+// of CTA r % grid waits until all partials of the pair are delivered, loads row r's
+// partials in a single round trip, merges them and counts the row as done.  The pass A
+// of the next wave sits between a pair's pass A and its pass B, so pass B's wait on
+// that count is normally already satisfied.
 //
 // Warp roles in a CTA of 512 threads: warp 0 issues TMA loads, warp 1 owns the
-// tensor-memory allocation and issues the MMAs, warps 4..15 are three independent
+// tensor-memory allocation and issues the MMAs, warp 2 merges rows, warps 4..15 are three independent
 // groups of four "statistics" warps that take accumulator tiles round-robin; a group
 // synchronises only with itself and writes its own partial results.  Every wait
 // (mbarrier or flag) is bounded; a timed-out wait raises CAKE_ERR_TIMEOUT and the CTA
@@ -56,15 +58,16 @@ struct TcParams {
   const ReqInfo* reqs;
   const int32_t* pair_aseg;     // [pairs + 1] pass-A segment ranges per pair
   uint32_t* pair_cnt;           // [pairs] delivered pass-A partials (monotonic over layers)
-  uint32_t* pair_flag;          // [pairs] epoch of the last published denominators (or null)
+  uint32_t* pair_done;          // [pairs] merged rows (monotonic over layers); null = pass B only
   float* lse2;                  // [pair][128] in tile row order r' = i*G + h
   float4* rowpart;              // pass A out: [A-segment][group][128] (m, z_all, z_win, w)
   float* raw;                   // pass B out: [H_kv][T]
   float* colpart;               // pass B out: [B-segment][group][G][2]
-  double* hhead;                // [req][H_q] entropy per query head
+  float* hrow;                  // [pair][128] sum_j p log2 p of every window row
   int32_t* status;
   int64_t T;
   uint32_t epoch;
+  int n_pairs;
   int Hkv, Hq, Sw, rows, d;
   float scale2, gamma, bessel;
 };
@@ -185,9 +188,6 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_release(uint32_t* p, uint32_t v) {
-  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
 
 struct Smem {
   uint8_t* q;          // 2 buffers x (2 slabs x 128 rows x 128 B)
@@ -199,8 +199,7 @@ struct Smem {
   uint64_t* q_full;    // [2]
   uint64_t* q_empty;   // [2]
   uint32_t* tmem_holder;
-  uint32_t* last_flag; // [NWG]
-  float* lse;          // [NWG][128]  per group: denominators (pass B) / row exchange (merge)
+  float* lse;          // [NWG][128]  per group: denominators of the pair in pass B
   float* red;          // [NWG][4 warps][16]
 };
 
@@ -220,7 +219,6 @@ __device__ __forceinline__ Smem carve(uint8_t* base) {
   s.q_full = (uint64_t*)p;    p += 16;
   s.q_empty = (uint64_t*)p;   p += 16;
   s.tmem_holder = (uint32_t*)p; p += 16;
-  s.last_flag = (uint32_t*)p;   p += 16;
   p = (uint8_t*)(((uintptr_t)p + 15) & ~(uintptr_t)15);
   s.lse = (float*)p;          p += NWG * 128 * 4;
   s.red = (float*)p;
@@ -355,6 +353,60 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         umma_commit(&S.q_empty[qb]);     // query buffer free once every MMA of the op has run
       }
     }
+  } else if (warp == 2) {
+    // ------------------------------------------------ row merger
+    // Row r of every pair is merged by CTA r % gridDim.x: once all partials of the pair have
+    // been delivered, the warp loads the row's partials in one round trip, merges them in a
+    // fixed order and publishes the row's base-2 log-sum-exp and entropy term.
+    if (P.pair_done) {
+      bool ok = true;
+      for (int pair = 0; pair < P.n_pairs && ok; ++pair) {
+        const int s_lo = P.pair_aseg[pair] * NWG, s_hi = P.pair_aseg[pair + 1] * NWG;
+        bool waited = false;
+        for (int r = blockIdx.x; r < P.rows; r += gridDim.x) {
+          if (!waited) {
+            const uint32_t want = (uint32_t)(s_hi - s_lo) * P.epoch;
+            const long long t0 = clock64();
+            while (ld_acquire(&P.pair_cnt[pair]) < want) {
+              if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
+              __nanosleep(100);
+            }
+            if (!ok) break;
+            waited = true;
+          }
+          float4 acc = make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
+          for (int base = s_lo; base < s_hi; base += 32 * 16) {
+            float4 pv[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+              const int sg = base + u * 32 + lane;
+              pv[u] = sg < s_hi ? __ldcg(&P.rowpart[(size_t)sg * 128 + r])
+                                : make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 16; ++u) acc = merge_rows(acc, pv[u]);
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            float4 other;
+            other.x = __shfl_xor_sync(0xffffffffu, acc.x, o);
+            other.y = __shfl_xor_sync(0xffffffffu, acc.y, o);
+            other.z = __shfl_xor_sync(0xffffffffu, acc.z, o);
+            other.w = __shfl_xor_sync(0xffffffffu, acc.w, o);
+            // the lower lane's partial always goes first, so every lane gets the same result
+            acc = (lane & o) ? merge_rows(other, acc) : merge_rows(acc, other);
+          }
+          if (lane == 0) {
+            const float lz = log2f(acc.y);
+            __stcg(&P.lse2[(size_t)pair * 128 + r], acc.x + lz);
+            // sum_j p log2 p over the observed keys = (w - log2(z) * z_obs) / z
+            __stcg(&P.hrow[(size_t)pair * 128 + r], (acc.w - lz * (acc.y - acc.z)) / acc.y);
+            __threadfence();
+            atomicAdd(&P.pair_done[pair], 1u);
+          }
+        }
+      }
+    }
   } else if (warp >= 4) {
     // ------------------------------------------------ statistics warps
     const int wg = (warp - 4) >> 2;                 // 0..NWG-1: takes tiles t with t % NWG == wg
@@ -373,9 +425,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const int pair = op.req * P.Hkv + op.g;
       if (op.phase) {
         // ---------------- pass B: thread = key, columns = rows r' = i*G + h
-        if (lane_row == 0 && P.pair_flag) {         // denominators of this pair published?
+        if (lane_row == 0 && P.pair_done) {         // every row's denominator published?
           const long long t0 = clock64();
-          while (ld_acquire(&P.pair_flag[pair]) != P.epoch) {
+          const uint32_t want = (uint32_t)P.rows * P.epoch;
+          while (ld_acquire(&P.pair_done[pair]) < want) {
             if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); break; }
             __nanosleep(32);
           }
@@ -536,45 +589,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         __stcg(&P.rowpart[((size_t)op.seg * NWG + wg) * 128 + lane_row], make_float4(m, z, zwin, w));
         __threadfence();
         named_bar(bar_wg, 128);
-        if (lane_row == 0) {
-          const uint32_t nseg = (uint32_t)(P.pair_aseg[pair + 1] - P.pair_aseg[pair]) * NWG;
-          const uint32_t old = atomicAdd(&P.pair_cnt[pair], 1u);
-          S.last_flag[wg] = (old + 1u == nseg * P.epoch) ? 1u : 0u;
-        }
-        named_bar(bar_wg, 128);
-        if (S.last_flag[wg]) {
-          // the pair's last partial: merge them all and publish the denominators
-          __threadfence();
-          const float4 none = make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
-          float4 part[4] = {none, none, none, none};
-          const int s_lo = P.pair_aseg[pair] * NWG, s_hi = P.pair_aseg[pair + 1] * NWG;
-          for (int sg = s_lo; sg < s_hi; sg += 8) {           // eight loads in flight per thread
-            float4 pv[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-              pv[u] = sg + u < s_hi ? __ldcg(&P.rowpart[(size_t)(sg + u) * 128 + lane_row]) : none;
-#pragma unroll
-            for (int u = 0; u < 8; ++u) part[u & 3] = merge_rows(part[u & 3], pv[u]);
-          }
-          const float4 tot = merge_rows(merge_rows(part[0], part[1]), merge_rows(part[2], part[3]));
-          float hrow = 0.f;
-          if (lane_row < P.rows) {
-            const float lz = log2f(tot.y);
-            __stcg(&P.lse2[(size_t)pair * 128 + lane_row], tot.x + lz);
-            // sum_j p log2 p over the observed keys = (w - log2(z) * z_obs) / z
-            hrow = (tot.w - lz * (tot.y - tot.z)) / tot.y;
-          }
-          lse_wg[lane_row] = hrow;
-          named_bar(bar_wg, 128);
-          if (lane_row < G) {                        // head h = rows h, h+G, h+2G, ...
-            double acc2 = 0.0;
-            for (int i = lane_row; i < P.rows; i += G) acc2 += (double)lse_wg[i];
-            P.hhead[(size_t)op.req * P.Hq + op.g * G + lane_row] = -0.6931471805599453 * acc2;
-          }
-          __threadfence();
-          named_bar(bar_wg, 128);
-          if (lane_row == 0) st_release(&P.pair_flag[pair], P.epoch);
-        }
+        if (lane_row == 0) atomicAdd(&P.pair_cnt[pair], 1u);
       }
     }
   }
@@ -806,7 +821,8 @@ int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const f
   P.rowpart = ctx->d_tc_rowpart;
   P.raw = ctx->d_raw;
   P.colpart = ctx->d_colpart;
-  P.hhead = ctx->d_hhead;
+  P.hrow = ctx->d_hrow;
+  P.n_pairs = n_pairs;
   P.status = ctx->d_status;
   P.T = ctx->total_tokens;
   P.Hkv = c.n_kv_heads; P.Hq = c.n_q_heads; P.Sw = c.window; P.rows = ctx->rows; P.d = c.head_dim;
@@ -823,12 +839,12 @@ int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const f
     count_launch();
     ctx->hhead_from_rows = false;
     P.cta_op = cta_full + (ctx->n_sm + 1);
-    P.pair_flag = nullptr;
+    P.pair_done = nullptr;
     P.epoch = 0;
   } else {
     ctx->hhead_from_rows = true;
     P.cta_op = cta_full;
-    P.pair_flag = ctx->d_tc_sync + ctx->max_pairs;
+    P.pair_done = ctx->d_tc_sync + ctx->max_pairs;
     P.epoch = ++ctx->tc_epoch;
   }
   cudaError_t e;
