@@ -156,7 +156,7 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
     x->max_tc_ops = (int32_t)(3 * segs + 8);
   }
   {
-    const size_t a = (size_t)x->max_units * c.n_kv_heads, b = (size_t)x->max_tc_segs * kScoreGroups;
+    const size_t a = (size_t)x->max_units * c.n_kv_heads, b = (size_t)x->max_tc_segs * kScoreWarps;
     ok = ok && dev_alloc(&x->d_colpart, (a > b ? a : b) * G * 2) == cudaSuccess;
   }
   if (x->use_tc) {

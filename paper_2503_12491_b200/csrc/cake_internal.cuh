@@ -13,6 +13,7 @@ constexpr int kMaxRows = 128;        // G * S_w rows handled per KV head
 constexpr int kSimtTileKeys = 64;    // keys per tile of the SIMT score kernels
 constexpr int kSimtThreads = 256;
 constexpr int kScoreGroups = 3;      // statistics warp groups per CTA of the tensor-core score kernel
+constexpr int kScoreWarps = 4 * kScoreGroups;   // statistics warps: one column-pass partial each
 
 // One request of the current batch (device copy in ctx->d_req).
 struct ReqInfo {
@@ -39,12 +40,15 @@ struct ScoreUnit {
 // column statistics).  `seg` numbers the partial results the step writes (one per
 // statistics warp group).
 struct ScoreOp {
+  int64_t base;    // row of the pair's first key in the packed K: g * T + cu[req]
   int32_t req;
   int32_t g;
   int32_t key0;
   int32_t nkeys;
   int32_t phase;
   int32_t seg;
+  int32_t n;       // non-window keys of the request
+  int32_t pad;
 };
 
 struct LayerPtrs {

@@ -50,7 +50,7 @@ __global__ void finalize_layer(const float* __restrict__ colpart, const ReqInfo*
 }
 
 // Same for the tensor-core path: one warp per query head.  Variance partials are indexed
-// by (pass-B segment, statistics group); the entropy comes either from the row pass
+// by (pass-B segment, statistics warp); the entropy comes either from the row pass
 // (hrow: sum_j p log2 p of every window row, tile row order r' = i*G + h) or, when the
 // caller supplied the denominators, from the column pass partials.
 __device__ inline double warp_sum_f64(double v) {
@@ -74,7 +74,7 @@ __global__ void finalize_layer_tc(const float* __restrict__ colpart,
     const int g = h / G, hl = h - g * G;
     const int pair = req * Hkv + g;
     double a = 0.0, b = 0.0;
-    const int s_lo = pair_seg[pair] * kScoreGroups, s_hi = pair_seg[pair + 1] * kScoreGroups;
+    const int s_lo = pair_seg[pair] * kScoreWarps, s_hi = pair_seg[pair + 1] * kScoreWarps;
     for (int sg = s_lo + lane; sg < s_hi; sg += 32) {
       const float2 p = *reinterpret_cast<const float2*>(colpart + ((size_t)sg * G + hl) * 2);
       a += (double)p.x;

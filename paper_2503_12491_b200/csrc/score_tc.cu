@@ -24,10 +24,11 @@
 // of the next wave sits between a pair's pass A and its pass B, so pass B's wait on
 // that count is normally already satisfied.
 //
-// Warp roles in a CTA of 512 threads: warp 0 issues TMA loads, warp 1 owns the
-// tensor-memory allocation and issues the MMAs, warp 2 merges rows, warps 4..15 are three independent
-// groups of four "statistics" warps that take accumulator tiles round-robin; a group
-// synchronises only with itself and writes its own partial results.  Every wait
+// Warp roles in a CTA of 512 threads: warps 0..11 are "statistics" warps in three groups of
+// four (a group takes every third accumulator tile, a warp owns 32 of its TMEM lanes, works
+// alone and writes its own partial results), warp 12 issues TMA loads, warp 13 owns the
+// tensor-memory allocation and issues the MMAs, warp 14 merges rows, warp 15 stages the
+// denominators of the next pass-B op in shared memory.  Every wait
 // (mbarrier or flag) is bounded; a timed-out wait raises CAKE_ERR_TIMEOUT and the CTA
 // drains and exits.
 #include "cake_internal.cuh"
@@ -45,7 +46,10 @@ constexpr int STAGES = 4;            // K tiles in flight
 constexpr int NBUF = 4;              // accumulator buffers (4 x 128 of the 512 TMEM columns)
 constexpr int NWG = kScoreGroups;    // statistics warp groups
 constexpr int STAT_THREADS = NWG * 128;
-constexpr int TC_THREADS = 128 + STAT_THREADS;
+constexpr int TC_THREADS = STAT_THREADS + 128;  // + TMA, MMA, row-merger and denominator warps
+constexpr int WARP_TMA = NWG * 4, WARP_MMA = NWG * 4 + 1, WARP_MERGE = NWG * 4 + 2,
+              WARP_LSE = NWG * 4 + 3;
+constexpr int NSTATW = NWG * 4;      // statistics warps
 constexpr int SLAB_BYTES = TILE * 128;   // one 64-element slab of a 128-row tile
 constexpr long long kSpinLimit = 4000000000ll;   // cycles (~2 s) before a wait gives up
 constexpr float kLog2e = 1.4426950408889634f;
@@ -62,7 +66,7 @@ struct TcParams {
   float* lse2;                  // [pair][128] in tile row order r' = i*G + h
   float4* rowpart;              // pass A out: [A-segment][group][128] (m, z_all, z_win, w)
   float* raw;                   // pass B out: [H_kv][T]
-  float* colpart;               // pass B out: [B-segment][group][G][2]
+  float* colpart;               // pass B out: [B-segment][statistics warp][G][2]
   float* hrow;                  // [pair][128] sum_j p log2 p of every window row
   int32_t* status;
   int64_t T;
@@ -110,12 +114,24 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_
   }
   return true;
 }
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0,
-                                            int c1) {
+// 2-D tiled TMA load with an L2 eviction-priority hint (a policy made by createpolicy).
+__device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* map, uint64_t* bar,
+                                                 int c0, int c1, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "l"(policy)
       : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0,
                                             int c1, int c2, int c3) {
@@ -143,29 +159,27 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
                    smem_u32(bar))
                : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
-  uint32_t r[32];
+// Starts the load of 32 consecutive fp32 columns of this thread's TMEM lane; the registers
+// are valid only after tmem_ld_wait on the same array.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
-        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
-        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
-        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Waits for the thread's outstanding TMEM loads.  The registers pass through the statement so
+// that no use of them can be scheduled before it.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-__device__ __forceinline__ void named_bar(int id, int count) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
@@ -189,6 +203,10 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
   return v;
 }
 
+__device__ __forceinline__ void red_release_add(uint32_t* p, uint32_t v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
 struct Smem {
   uint8_t* q;          // 2 buffers x (2 slabs x 128 rows x 128 B)
   uint8_t* k;          // STAGES x (2 slabs x 128 rows x 128 B)
@@ -198,14 +216,17 @@ struct Smem {
   uint64_t* acc_empty; // [NBUF]
   uint64_t* q_full;    // [2]
   uint64_t* q_empty;   // [2]
+  uint64_t* lse_full;  // [2]
+  uint64_t* lse_free;  // [2]
   uint32_t* tmem_holder;
-  float* lse;          // [NWG][128]  per group: denominators of the pair in pass B
-  float* red;          // [NWG][4 warps][16]
+  float* lse;          // [2][128] denominators of the pairs of the current / next pass-B op
+  ScoreOp* ops;        // [kSmemOps] the first ops of this CTA's program
 };
 
 constexpr size_t kQBytes = 2 * SLAB_BYTES;
+constexpr int kSmemOps = 128;        // ops of a CTA's program kept in shared memory
 constexpr size_t kSmemBytes = 1024 /*align*/ + 2 * kQBytes + (size_t)STAGES * 2 * SLAB_BYTES + 256 +
-                              NWG * 128 * 4 + NWG * 64 * 4 + 64;
+                              2 * 128 * 4 + kSmemOps * sizeof(ScoreOp) + 64;
 
 __device__ __forceinline__ Smem carve(uint8_t* base) {
   Smem s;
@@ -218,10 +239,12 @@ __device__ __forceinline__ Smem carve(uint8_t* base) {
   s.acc_empty = (uint64_t*)p; p += 8 * NBUF;
   s.q_full = (uint64_t*)p;    p += 16;
   s.q_empty = (uint64_t*)p;   p += 16;
+  s.lse_full = (uint64_t*)p;  p += 16;
+  s.lse_free = (uint64_t*)p;  p += 16;
   s.tmem_holder = (uint32_t*)p; p += 16;
   p = (uint8_t*)(((uintptr_t)p + 15) & ~(uintptr_t)15);
-  s.lse = (float*)p;          p += NWG * 128 * 4;
-  s.red = (float*)p;
+  s.lse = (float*)p;          p += 2 * 128 * 4;
+  s.ops = (ScoreOp*)p;
   return s;
 }
 
@@ -257,13 +280,19 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     for (int i = 0; i < STAGES; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], 1); }
     for (int i = 0; i < NBUF; ++i) { mbar_init(&S.acc_full[i], 1); mbar_init(&S.acc_empty[i], 128); }
     for (int i = 0; i < 2; ++i) { mbar_init(&S.q_full[i], 1); mbar_init(&S.q_empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&S.lse_full[i], 1); mbar_init(&S.lse_free[i], NSTATW); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // the program of this CTA: a global read per op would put an L2 round trip on every op
+  for (int i = threadIdx.x; i < min(op_hi - op_lo, kSmemOps); i += TC_THREADS) S.ops[i] = P.ops[op_lo + i];
+  auto get_op = [&](int oi) -> ScoreOp {
+    return oi - op_lo < kSmemOps ? S.ops[oi - op_lo] : P.ops[oi];
+  };
   // rows of the query tiles that TMA never writes must read as zero
   for (int i = threadIdx.x; i < (int)(2 * kQBytes / 16); i += TC_THREADS)
     reinterpret_cast<uint4*>(S.q)[i] = make_uint4(0, 0, 0, 0);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  if (warp == 1) {
+  if (warp == WARP_MMA) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(S.tmem_holder)),
                  "r"(512)
@@ -275,17 +304,19 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = *S.tmem_holder;
 
-  if (warp == 0) {
+  if (warp == WARP_TMA) {
     // ------------------------------------------------ TMA producer
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&q_map) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
+      // pass A's tiles are read again by pass B: keep them in L2; pass B's read is the last
+      const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
       uint32_t t = 0, qn = 0;
       bool ok = true;
       for (int oi = op_lo; oi < op_hi && ok; ++oi) {
-        const ScoreOp op = P.ops[oi];
+        const ScoreOp op = get_op(oi);
         if (op.nkeys <= 0) continue;
-        const ReqInfo rq = P.reqs[op.req];
+        const uint64_t pol = (op.phase || !P.pair_done) ? drop : keep;
         const int qb = qn & 1;
         // the MMAs of the op that used this query buffer two ops ago must be done
         ok = mbar_wait(&S.q_empty[qb], ((qn >> 1) & 1) ^ 1, P.status);
@@ -295,7 +326,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         for (int sl = 0; sl < n_slab; ++sl)
           tma_load_4d(S.q + qb * kQBytes + sl * SLAB_BYTES, &q_map, &S.q_full[qb], sl * 64, op.g * G,
                       0, op.req);
-        const int64_t row0 = (int64_t)op.g * P.T + rq.cu + op.key0;
+        const int64_t row0 = op.base + op.key0;
         const int ntiles = (op.nkeys + TILE - 1) / TILE;
         for (int it = 0; it < ntiles; ++it, ++t) {
           const int s = t % STAGES;
@@ -304,7 +335,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           mbar_expect_tx(&S.full[s], stage_bytes);
           uint8_t* dst = S.k + (size_t)s * 2 * SLAB_BYTES;
           for (int sl = 0; sl < n_slab; ++sl)
-            tma_load_2d(dst + sl * SLAB_BYTES, &k_map, &S.full[s], sl * 64, (int)(row0 + it * TILE));
+            tma_load_2d_hint(dst + sl * SLAB_BYTES, &k_map, &S.full[s], sl * 64,
+                             (int)(row0 + it * TILE), pol);
         }
       }
       // do not leave the CTA while a bulk copy may still be writing its shared memory
@@ -314,13 +346,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       for (uint32_t u = qn > 2 ? qn - 2 : 0; u < qn; ++u)
         mbar_wait(&S.q_full[u & 1], (u >> 1) & 1, P.status);
     }
-  } else if (warp == 1) {
+  } else if (warp == WARP_MMA) {
     // ------------------------------------------------ MMA issuer
     if (lane == 0) {
       uint32_t t = 0, qn = 0;
       bool ok = true;
       for (int oi = op_lo; oi < op_hi && ok; ++oi) {
-        const ScoreOp op = P.ops[oi];
+        const ScoreOp op = get_op(oi);
         if (op.nkeys <= 0) continue;
         const uint32_t idesc = op.phase ? instr_desc(128, rows_pad) : instr_desc(128, TILE);
         const int qb = qn & 1;
@@ -353,7 +385,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         umma_commit(&S.q_empty[qb]);     // query buffer free once every MMA of the op has run
       }
     }
-  } else if (warp == 2) {
+  } else if (warp == WARP_MERGE) {
     // ------------------------------------------------ row merger
     // Row r of every pair is merged by CTA r % gridDim.x: once all partials of the pair have
     // been delivered, the warp loads the row's partials in one round trip, merges them in a
@@ -365,7 +397,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         bool waited = false;
         for (int r = blockIdx.x; r < P.rows; r += gridDim.x) {
           if (!waited) {
-            const uint32_t want = (uint32_t)(s_hi - s_lo) * P.epoch;
+            const uint32_t want = (uint32_t)(s_hi - s_lo) * 4u * P.epoch;   // one per warp
             const long long t0 = clock64();
             while (ld_acquire(&P.pair_cnt[pair]) < want) {
               if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
@@ -375,16 +407,16 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             waited = true;
           }
           float4 acc = make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
-          for (int base = s_lo; base < s_hi; base += 32 * 16) {
-            float4 pv[16];
+          for (int base = s_lo; base < s_hi; base += 32 * 8) {
+            float4 pv[8];
 #pragma unroll
-            for (int u = 0; u < 16; ++u) {
+            for (int u = 0; u < 8; ++u) {
               const int sg = base + u * 32 + lane;
               pv[u] = sg < s_hi ? __ldcg(&P.rowpart[(size_t)sg * 128 + r])
                                 : make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
             }
 #pragma unroll
-            for (int u = 0; u < 16; ++u) acc = merge_rows(acc, pv[u]);
+            for (int u = 0; u < 8; ++u) acc = merge_rows(acc, pv[u]);
           }
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) {
@@ -407,35 +439,56 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         }
       }
     }
-  } else if (warp >= 4) {
+  } else if (warp == WARP_LSE) {
+    // ------------------------------------------------ denominator fetcher
+    // For every pass-B op of this CTA, in program order: wait until all rows of the op's pair
+    // are merged, copy the pair's 128 denominators into a two-slot shared-memory ring.
+    uint32_t kb = 0;
+    bool ok = true;
+    for (int oi = op_lo; oi < op_hi && ok; ++oi) {
+      const ScoreOp op = get_op(oi);
+      if (op.nkeys <= 0 || !op.phase) continue;
+      const int slot = kb & 1;
+      const int pair = op.req * P.Hkv + op.g;
+      if (lane == 0) {
+        ok = mbar_wait(&S.lse_free[slot], ((kb >> 1) & 1) ^ 1, P.status);
+        if (ok && P.pair_done) {
+          const uint32_t want = (uint32_t)P.rows * P.epoch;
+          const long long t0 = clock64();
+          while (ld_acquire(&P.pair_done[pair]) < want) {
+            if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
+            __nanosleep(64);
+          }
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(P.lse2 + (size_t)pair * 128) + lane);
+      reinterpret_cast<float4*>(S.lse + slot * 128)[lane] = v;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&S.lse_full[slot]);
+      ++kb;
+    }
+  } else {
     // ------------------------------------------------ statistics warps
-    const int wg = (warp - 4) >> 2;                 // 0..NWG-1: takes tiles t with t % NWG == wg
+    // Every warp works alone: it owns TMEM lanes 32*quad.. of the tiles its group takes, writes
+    // its own partial results and never waits for another statistics warp.
+    const int wg = warp >> 2;                       // takes tiles t with t % NWG == wg
     const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
     const int lane_row = quad * 32 + lane;          // accumulator lane (row in pass A, key in pass B)
-    const int bar_wg = 1 + wg;                      // named barrier of this warp group
-    float* lse_wg = S.lse + wg * 128;
-    float* red_wg = S.red + wg * 64;
-    uint32_t t = 0;
+    uint32_t t = 0, kb = 0;
     bool ok = true;
     for (int oi = op_lo; oi < op_hi; ++oi) {
-      const ScoreOp op = P.ops[oi];
+      const ScoreOp op = get_op(oi);
       if (op.nkeys <= 0) continue;
-      const ReqInfo rq = P.reqs[op.req];
       const int ntiles = (op.nkeys + TILE - 1) / TILE;
       const int pair = op.req * P.Hkv + op.g;
       if (op.phase) {
         // ---------------- pass B: thread = key, columns = rows r' = i*G + h
-        if (lane_row == 0 && P.pair_done) {         // every row's denominator published?
-          const long long t0 = clock64();
-          const uint32_t want = (uint32_t)P.rows * P.epoch;
-          while (ld_acquire(&P.pair_done[pair]) < want) {
-            if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); break; }
-            __nanosleep(32);
-          }
-        }
-        named_bar(bar_wg, 128);
-        lse_wg[lane_row] = lane_row < P.rows ? __ldcg(&P.lse2[(size_t)pair * 128 + lane_row]) : 0.f;
-        named_bar(bar_wg, 128);
+        const int slot = kb & 1;
+        if (ok) ok = mbar_wait(&S.lse_full[slot], (kb >> 1) & 1, P.status);
+        ++kb;
+        const float* lse_s = S.lse + slot * 128;
         float vacc[G], hs[G];
 #pragma unroll
         for (int h = 0; h < G; ++h) { vacc[h] = 0.f; hs[h] = 0.f; }
@@ -451,15 +504,17 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 #pragma unroll
           for (int h = 0; h < G; ++h) { s1[h] = 0.f; s2[h] = 0.f; hk[h] = 0.f; }
           for (int c0 = 0; c0 < P.rows; c0 += 32) {
-            float v[32];
-            tmem_ld32(taddr + c0, v);
+            uint32_t r[32];
+            tmem_ld32_issue(taddr + c0, r);
+            tmem_ld_wait(r);
+            if (c0 + 32 >= P.rows) { tc_fence_before(); mbar_arrive(&S.acc_empty[b]); }
             // 32 columns = 32/G window rows x G heads
 #pragma unroll
             for (int ii = 0; ii < 32 / G; ++ii) {
               float a = 0.f;
 #pragma unroll
               for (int h = 0; h < G; ++h) {
-                const float tt = fmaf(v[ii * G + h], P.scale2, -lse_wg[c0 + ii * G + h]);
+                const float tt = fmaf(__uint_as_float(r[ii * G + h]), P.scale2, -lse_s[c0 + ii * G + h]);
                 const float p = ex2(tt);
                 s1[h] += p;
                 s2[h] = fmaf(p, p, s2[h]);
@@ -469,10 +524,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
               a2 = fmaf(a, a, a2);
             }
           }
-          tc_fence_before();
-          mbar_arrive(&S.acc_empty[b]);
           const int j = op.key0 + it * TILE + lane_row;          // key index inside the request
-          if (j < rq.n && it * TILE + lane_row < op.nkeys) {
+          if (j < op.n && it * TILE + lane_row < op.nkeys) {
             float a1 = 0.f;
 #pragma unroll
             for (int h = 0; h < G; ++h) {
@@ -483,36 +536,30 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
             const float mean = a1 * inv_g * inv_sw;
             const float var = fmaxf(a2 * inv_g * inv_g * inv_sw - mean * mean, 0.f) * P.bessel;
-            P.raw[(size_t)op.g * P.T + rq.cu + j] = fmaf(P.gamma, var, mean);
+            P.raw[op.base + j] = fmaf(P.gamma, var, mean);
           }
         }
-        // fixed-order reduction over the group's threads
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&S.lse_free[slot]);          // done with this op's denominators
+        // fixed-order reduction over the warp's keys
 #pragma unroll
         for (int h = 0; h < G; ++h) {
           float x = vacc[h], y = hs[h];
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) {
             x += __shfl_xor_sync(0xffffffffu, x, o);
-            y += __shfl_xor_sync(0xffffffffu, y, o);
+            if (kEntropyB) y += __shfl_xor_sync(0xffffffffu, y, o);
           }
-          if (lane == 0) { red_wg[quad * 16 + h] = x; red_wg[quad * 16 + 8 + h] = y; }
-        }
-        named_bar(bar_wg, 128);
-        if (lane_row < G) {
-          float acc = 0.f, hacc = 0.f;
-#pragma unroll
-          for (int w2 = 0; w2 < 4; ++w2) {
-            acc += red_wg[w2 * 16 + lane_row];
-            hacc += red_wg[w2 * 16 + 8 + lane_row];
+          if (lane == h) {
+            float* dst = P.colpart + (((size_t)op.seg * NSTATW + warp) * G + h) * 2;
+            dst[0] = y;
+            dst[1] = x;
           }
-          float* dst = P.colpart + (((size_t)op.seg * NWG + wg) * G + lane_row) * 2;
-          dst[0] = hacc;
-          dst[1] = acc;
         }
       } else {
         // ---------------- pass A: thread = window row r' = i*G + h, columns = keys
         const int i_row = lane_row / G;
-        const int last = rq.n + i_row;                 // last key this row may attend to
+        const int last = op.n + i_row;                 // last key this row may attend to
         float m = -CUDART_INF_F, z = 0.f, zwin = 0.f, w = 0.f;
         for (int it = 0; it < ntiles; ++it, ++t) {
           if ((int)(t % NWG) != wg) continue;
@@ -522,15 +569,18 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           tc_fence_after();
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * 128);
           const int key0 = op.key0 + it * TILE;
-          const bool interior = key0 + TILE <= rq.n && it * TILE + TILE <= op.nkeys;
+          const bool interior = key0 + TILE <= op.n && it * TILE + TILE <= op.nkeys;
 #pragma unroll 1
           for (int c0 = 0; c0 < TILE; c0 += 32) {
-            float v[32];
-            tmem_ld32(taddr + c0, v);
+            uint32_t r[32];
+            tmem_ld32_issue(taddr + c0, r);
+            tmem_ld_wait(r);
+            if (c0 + 32 >= TILE) { tc_fence_before(); mbar_arrive(&S.acc_empty[b]); }
             if (interior) {
-              float c4[4] = {v[0], v[1], v[2], v[3]};
+              float c4[4] = {__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]),
+                             __uint_as_float(r[3])};
 #pragma unroll
-              for (int e = 4; e < 32; ++e) c4[e & 3] = fmaxf(c4[e & 3], v[e]);
+              for (int e = 4; e < 32; ++e) c4[e & 3] = fmaxf(c4[e & 3], __uint_as_float(r[e]));
               const float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3])) * P.scale2;
               if (cm > m + kLazyMax) {                        // rare after the first tiles
                 const float mn = cm;
@@ -543,7 +593,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
               float zc[4] = {0.f, 0.f, 0.f, 0.f}, wc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
-                const float tt = fmaf(v[e], P.scale2, -m);
+                const float tt = fmaf(__uint_as_float(r[e]), P.scale2, -m);
                 const float ee = ex2(tt);
                 zc[e & 3] += ee;
                 wc[e & 3] = fmaf(ee, tt, wc[e & 3]);
@@ -556,7 +606,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
               for (int e = 0; e < 32; ++e) {
                 const int j = key0 + c0 + e;
                 const bool vis = (it * TILE + c0 + e < op.nkeys) && j <= last;
-                cm = vis ? fmaxf(cm, v[e]) : cm;
+                cm = vis ? fmaxf(cm, __uint_as_float(r[e])) : cm;
               }
               if (cm != -CUDART_INF_F) {
                 cm *= P.scale2;
@@ -572,8 +622,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 for (int e = 0; e < 32; ++e) {
                   const int j = key0 + c0 + e;
                   const bool vis = (it * TILE + c0 + e < op.nkeys) && j <= last;
-                  const bool obs = j < rq.n;
-                  const float tt = fmaf(v[e], P.scale2, -m);
+                  const bool obs = j < op.n;
+                  const float tt = fmaf(__uint_as_float(r[e]), P.scale2, -m);
                   const float ee = vis ? ex2(tt) : 0.f;
                   z += ee;
                   zwin += obs ? 0.f : ee;
@@ -582,21 +632,19 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
               }
             }
           }
-          tc_fence_before();
-          mbar_arrive(&S.acc_empty[b]);
         }
-        // deliver this group's partial rows of the segment
+        // deliver this warp's 32 partial rows of the segment; the release orders them before
+        // the count without stalling the warp
         __stcg(&P.rowpart[((size_t)op.seg * NWG + wg) * 128 + lane_row], make_float4(m, z, zwin, w));
-        __threadfence();
-        named_bar(bar_wg, 128);
-        if (lane_row == 0) atomicAdd(&P.pair_cnt[pair], 1u);
+        __syncwarp();
+        if (lane == 0) red_release_add(&P.pair_cnt[pair], 1u);
       }
     }
   }
   // ------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == WARP_MMA) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512)
                  : "memory");
@@ -655,7 +703,8 @@ cudaError_t launch_g(bool entropy_b, int n_cta, cudaStream_t st, const CUtensorM
 // of a wave of `W` tiles shared by `n_cta` CTAs (slot c owns flat tiles
 // [c*W/n_cta, (c+1)*W/n_cta)), into per-slot segments; slot c belongs to CTA (c+rot)%n_cta.
 void cut_pair(std::vector<std::vector<ScoreOp>>& per_cta, int rot, int n_cta, int64_t W, int64_t flat,
-              int tiles, int keys, int req, int g, int phase, int32_t& seg_counter) {
+              int tiles, int keys, int req, int g, int phase, int32_t& seg_counter, int64_t base,
+              int n_obs) {
   int t0 = 0;
   while (t0 < tiles) {
     const int64_t f = flat + t0;
@@ -665,6 +714,7 @@ void cut_pair(std::vector<std::vector<ScoreOp>>& per_cta, int rot, int n_cta, in
     const int64_t share_end = (int64_t)(c + 1) * W / n_cta;
     const int t1 = (int)((share_end - flat) < tiles ? (share_end - flat) : tiles);
     ScoreOp op;
+    op.base = base; op.n = n_obs; op.pad = 0;
     op.req = req; op.g = g; op.key0 = t0 * TILE;
     const int kend = t1 * TILE < keys ? t1 * TILE : keys;
     op.nkeys = kend - t0 * TILE;
@@ -701,6 +751,7 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
   const cake_config& c = ctx->cfg;
   const int Hkv = c.n_kv_heads;
   const int n_pairs = n_req * Hkv;
+  const int64_t T = n_req > 0 ? ctx->h_req[n_req - 1].cu + ctx->h_req[n_req - 1].N : 0;
   int64_t tilesA_total = 0;
   for (int r = 0; r < n_req; ++r) tilesA_total += (int64_t)Hkv * ((ctx->h_req[r].N + TILE - 1) / TILE);
   const int n_cta = (int)(tilesA_total < ctx->n_sm ? tilesA_total : ctx->n_sm);
@@ -737,12 +788,14 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
       const int ta = (rq.N + TILE - 1) / TILE, tb = (rq.n + TILE - 1) / TILE;
       pair_aseg[p] = aseg;
       pair_bseg[p] = bseg;
-      cut_pair(wa, rot, n_cta, WA, fa, ta, rq.N, r, g, 0, aseg);
+      const int64_t base = (int64_t)g * T + rq.cu;
+      cut_pair(wa, rot, n_cta, WA, fa, ta, rq.N, r, g, 0, aseg, base, rq.n);
       // pass B walks the same flat tile positions, so a CTA re-reads the tiles it brought in
-      if (tb > 0) cut_pair(wb, rot, n_cta, WA, fa, tb, rq.n, r, g, 1, bseg);
+      if (tb > 0) cut_pair(wb, rot, n_cta, WA, fa, tb, rq.n, r, g, 1, bseg, base, rq.n);
       fa += ta;
     }
-    rot = (rot + 37) % n_cta;             // a wave's remainder tiles land on different CTAs each time
+    // a wave's remainder tiles land on different CTAs each time (golden-ratio stride)
+    rot = (rot + (int)(n_cta * 0.381966) + 1) % n_cta;
     for (int cta = 0; cta < n_cta; ++cta) {
       full[cta].insert(full[cta].end(), wa[cta].begin(), wa[cta].end());
       if (wv > 0) full[cta].insert(full[cta].end(), wb_prev[cta].begin(), wb_prev[cta].end());
