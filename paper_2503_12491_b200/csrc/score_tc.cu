@@ -43,7 +43,8 @@ namespace {
 
 constexpr int TILE = 128;            // keys per tile
 constexpr int STAGES = 4;            // K tiles in flight
-constexpr int NBUF = 4;              // accumulator buffers (4 x 128 of the 512 TMEM columns)
+constexpr int NBUF = 3;              // accumulator buffers: 3 x 128 of the 512 TMEM columns
+constexpr int TMEM_Q_COL = NBUF * 128;   // + 64 columns: the window queries as pass A's A operand
 constexpr int NWG = kScoreGroups;    // statistics warp groups
 constexpr int STAT_THREADS = NWG * 128;
 constexpr int TC_THREADS = STAT_THREADS + 128;  // + TMA, MMA, row-merger and denominator warps
@@ -146,13 +147,32 @@ __device__ __forceinline__ void tc_fence_before() {
 __device__ __forceinline__ void tc_fence_after() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
-                                          uint32_t idesc, uint32_t accumulate) {
+// The issuing thread is a single lane whose dependent instructions run at a few cycles each, so
+// the per-MMA work is kept minimal: descriptors differ only in the 14-bit address field of their
+// low word, the high word (stride, version, swizzle) is a constant, and the accumulate flag is
+// an immediate.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // SBO, version 1, SWIZZLE_128B
+template <int kAcc>
+__device__ __forceinline__ void umma_ss(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
   asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      "{\n.reg .pred p;\n.reg .b64 da, db;\nsetp.ne.b32 p, %4, 0;\n"
+      "mov.b64 da, {%1, %5};\nmov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n}"
+      ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "n"(kAcc), "r"(kDescHi)
       : "memory");
+}
+template <int kAcc>
+__device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t idesc) {
+  asm volatile(
+      "{\n.reg .pred p;\n.reg .b64 db;\nsetp.ne.b32 p, %4, 0;\n"
+      "mov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n}"
+      ::"r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(idesc), "n"(kAcc), "r"(kDescHi)
+      : "memory");
+}
+// Copies 128 rows x 32 bytes (one K = 16 slice of a K-major operand) from shared to tensor memory.
+__device__ __forceinline__ void tmem_cp_128x256b(uint32_t tmem_dst, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(tmem_dst), "l"(sdesc) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
@@ -278,7 +298,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], 1); }
-    for (int i = 0; i < NBUF; ++i) { mbar_init(&S.acc_full[i], 1); mbar_init(&S.acc_empty[i], 128); }
+    for (int i = 0; i < NBUF; ++i) { mbar_init(&S.acc_full[i], 1); mbar_init(&S.acc_empty[i], 4); }
     for (int i = 0; i < 2; ++i) { mbar_init(&S.q_full[i], 1); mbar_init(&S.q_empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&S.lse_full[i], 1); mbar_init(&S.lse_free[i], NSTATW); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -350,6 +370,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     // ------------------------------------------------ MMA issuer
     if (lane == 0) {
       uint32_t t = 0, qn = 0;
+      const uint32_t k_lo0 = (smem_u32(S.k) & 0x3FFFFu) >> 4;
       bool ok = true;
       for (int oi = op_lo; oi < op_hi && ok; ++oi) {
         const ScoreOp op = get_op(oi);
@@ -360,6 +381,19 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         ++qn;
         if (!ok) break;
         const uint32_t qaddr = smem_u32(S.q + qb * kQBytes);
+        const uint32_t q_lo = (qaddr & 0x3FFFFu) >> 4;      // address field of the descriptors
+        const uint32_t tmem_q = tmem_base + (uint32_t)TMEM_Q_COL;
+        if (!op.phase) {
+          // pass A multiplies every key tile by the same queries: hold them in tensor memory, so
+          // that an MMA reads only the key tile from shared memory.  The copies run in issue
+          // order behind the previous op's MMAs and ahead of this op's.
+          tc_fence_after();
+          for (int sl = 0; sl < n_slab; ++sl)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              tmem_cp_128x256b(tmem_q + (uint32_t)((sl * 4 + ks) * 8),
+                               smem_desc(qaddr + sl * SLAB_BYTES + ks * 32));
+        }
         const int ntiles = (op.nkeys + TILE - 1) / TILE;
         for (int it = 0; it < ntiles; ++it, ++t) {
           const int s = t % STAGES, b = t % NBUF;
@@ -368,15 +402,33 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           ok = mbar_wait(&S.full[s], (t / STAGES) & 1, P.status);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t kaddr = smem_u32(S.k + (size_t)s * 2 * SLAB_BYTES);
+          const uint32_t k_lo = k_lo0 + (uint32_t)s * (uint32_t)((2 * SLAB_BYTES) >> 4);
           const uint32_t tmem_d = tmem_base + (uint32_t)(b * 128);
-          for (int sl = 0; sl < n_slab; ++sl) {
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-              const uint64_t kd = smem_desc(kaddr + sl * SLAB_BYTES + ks * 32);
-              const uint64_t qd = smem_desc(qaddr + sl * SLAB_BYTES + ks * 32);
-              if (op.phase) umma_bf16(tmem_d, kd, qd, idesc, (sl | ks) != 0);
-              else          umma_bf16(tmem_d, qd, kd, idesc, (sl | ks) != 0);
+          if (op.phase) {
+            // D[key][row] = K Q^T
+            umma_ss<0>(tmem_d, k_lo, q_lo, idesc);
+            umma_ss<1>(tmem_d, k_lo + 2, q_lo + 2, idesc);
+            umma_ss<1>(tmem_d, k_lo + 4, q_lo + 4, idesc);
+            umma_ss<1>(tmem_d, k_lo + 6, q_lo + 6, idesc);
+            if (n_slab == 2) {
+              constexpr uint32_t o = SLAB_BYTES >> 4;
+              umma_ss<1>(tmem_d, k_lo + o, q_lo + o, idesc);
+              umma_ss<1>(tmem_d, k_lo + o + 2, q_lo + o + 2, idesc);
+              umma_ss<1>(tmem_d, k_lo + o + 4, q_lo + o + 4, idesc);
+              umma_ss<1>(tmem_d, k_lo + o + 6, q_lo + o + 6, idesc);
+            }
+          } else {
+            // D[row][key] = Q K^T, queries from tensor memory
+            umma_ts<0>(tmem_d, tmem_q, k_lo, idesc);
+            umma_ts<1>(tmem_d, tmem_q + 8, k_lo + 2, idesc);
+            umma_ts<1>(tmem_d, tmem_q + 16, k_lo + 4, idesc);
+            umma_ts<1>(tmem_d, tmem_q + 24, k_lo + 6, idesc);
+            if (n_slab == 2) {
+              constexpr uint32_t o = SLAB_BYTES >> 4;
+              umma_ts<1>(tmem_d, tmem_q + 32, k_lo + o, idesc);
+              umma_ts<1>(tmem_d, tmem_q + 40, k_lo + o + 2, idesc);
+              umma_ts<1>(tmem_d, tmem_q + 48, k_lo + o + 4, idesc);
+              umma_ts<1>(tmem_d, tmem_q + 56, k_lo + o + 6, idesc);
             }
           }
           umma_commit(&S.empty[s]);
@@ -507,14 +559,24 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             uint32_t r[32];
             tmem_ld32_issue(taddr + c0, r);
             tmem_ld_wait(r);
-            if (c0 + 32 >= P.rows) { tc_fence_before(); mbar_arrive(&S.acc_empty[b]); }
+            if (c0 + 32 >= P.rows) {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&S.acc_empty[b]);
+            }
             // 32 columns = 32/G window rows x G heads
+            float ls[32];
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) {
+              const float4 l4 = reinterpret_cast<const float4*>(lse_s + c0)[q4];
+              ls[q4 * 4 + 0] = l4.x; ls[q4 * 4 + 1] = l4.y; ls[q4 * 4 + 2] = l4.z; ls[q4 * 4 + 3] = l4.w;
+            }
 #pragma unroll
             for (int ii = 0; ii < 32 / G; ++ii) {
               float a = 0.f;
 #pragma unroll
               for (int h = 0; h < G; ++h) {
-                const float tt = fmaf(__uint_as_float(r[ii * G + h]), P.scale2, -lse_s[c0 + ii * G + h]);
+                const float tt = fmaf(__uint_as_float(r[ii * G + h]), P.scale2, -ls[ii * G + h]);
                 const float p = ex2(tt);
                 s1[h] += p;
                 s2[h] = fmaf(p, p, s2[h]);
@@ -575,7 +637,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             uint32_t r[32];
             tmem_ld32_issue(taddr + c0, r);
             tmem_ld_wait(r);
-            if (c0 + 32 >= TILE) { tc_fence_before(); mbar_arrive(&S.acc_empty[b]); }
+            if (c0 + 32 >= TILE) {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&S.acc_empty[b]);
+            }
             if (interior) {
               float c4[4] = {__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]),
                              __uint_as_float(r[3])};
