@@ -60,7 +60,10 @@ void free_ctx(cake_ctx* c) {
   if (!c) return;
   cudaFree(c->d_req); cudaFree(c->d_units); cudaFree(c->d_H); cudaFree(c->d_V); cudaFree(c->d_P);
   cudaFree(c->d_budget[0]); cudaFree(c->d_budget[1]); cudaFree(c->d_status); cudaFree(c->d_raw);
-  cudaFree(c->d_fresh); cudaFree(c->list_vals); cudaFree(c->list_pos); cudaFree(c->d_lse2);
+  cudaFree(c->d_fresh); cudaFree(c->d_lists); cudaFree(c->d_prefix); cudaFree(c->d_lstate);
+  cudaFree(c->d_hist); cudaFree(c->d_fill); cudaFree(c->d_arrivals); cudaFree(c->d_chunks);
+  cudaFree(c->d_pos_packed); cudaFree(c->d_bitmap); cudaFree(c->d_lse2);
+  if (c->h_chunks) cudaFreeHost(c->h_chunks);
   cudaFree(c->d_rowpart); cudaFree(c->d_colpart);
   cudaFree(c->d_tc_ops); cudaFree(c->d_tc_index); cudaFree(c->d_tc_sync);
   cudaFree(c->d_tc_rowpart); cudaFree(c->d_lse2_tc); cudaFree(c->d_hrow);
@@ -122,8 +125,18 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   const int64_t R = c.max_requests;
   // a unit never spans requests: at most T/64 + R units
   x->max_units = (int32_t)(T / kSimtTileKeys + R + 1);
-  int64_t list_tokens = R * x->sel_budget < T ? R * x->sel_budget : T;
-  x->list_elems = list_tokens * c.n_layers * c.n_kv_heads;
+  x->list_elems = T * c.n_layers * c.n_kv_heads;
+  x->max_lists = R * c.n_layers * c.n_kv_heads;
+  x->max_chunks = (int32_t)(T / kChunkKeys + R + 1);
+  {
+    // packed rows: H_kv * sum_r min(B_total, L * N_r) <= H_kv * min(R * B_total, L * T)
+    const int64_t a = R * c.total_budget, b = (int64_t)c.n_layers * T;
+    x->pos_packed_cap = (int64_t)c.n_kv_heads * (a < b ? a : b);
+    // a request longer than the shared-memory bitmap orders its positions in global scratch:
+    // one bitmap of ceil(n/32) words per (request, layer, head) list
+    x->bitmap_words = T > (int64_t)kBitmapSmemWords * 32
+                          ? (int64_t)c.n_layers * c.n_kv_heads * (T / 32 + R + 1) : 0;
+  }
   x->h_cu = (int64_t*)calloc((size_t)R + 1, sizeof(int64_t));
   bool ok = x->h_cu != nullptr;
   ok = ok && cudaMallocHost((void**)&x->h_req, sizeof(ReqInfo) * R) == cudaSuccess;
@@ -139,8 +152,19 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   ok = ok && dev_alloc(&x->d_status, 1) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_raw, (size_t)c.n_kv_heads * T) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_fresh, (size_t)c.n_kv_heads * T) == cudaSuccess;
-  ok = ok && dev_alloc(&x->list_vals, (size_t)x->list_elems) == cudaSuccess;
-  ok = ok && dev_alloc(&x->list_pos, (size_t)x->list_elems) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_lists, (size_t)x->list_elems) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_prefix, (size_t)x->max_lists * (kBins + 1)) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_lstate, (size_t)x->max_lists) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_hist, (size_t)R * c.n_kv_heads * kBins) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_fill, (size_t)R * c.n_kv_heads * kBins) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_arrivals, (size_t)R * c.n_kv_heads) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_chunks, (size_t)x->max_chunks) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_pos_packed, (size_t)x->pos_packed_cap) == cudaSuccess;
+  if (x->bitmap_words > 0) ok = ok && dev_alloc(&x->d_bitmap, (size_t)x->bitmap_words) == cudaSuccess;
+  ok = ok && cudaMallocHost((void**)&x->h_chunks, sizeof(ScoreUnit) * x->max_chunks) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_hist, 0, sizeof(uint32_t) * R * c.n_kv_heads * kBins) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_fill, 0, sizeof(uint32_t) * R * c.n_kv_heads * kBins) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_arrivals, 0, sizeof(uint32_t) * R * c.n_kv_heads) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_lse2, (size_t)R * c.n_q_heads * c.window) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_rowpart, (size_t)x->max_units * c.n_kv_heads * x->rows) == cudaSuccess;
   {
@@ -209,7 +233,7 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
       ctx->upload_pending = false;
     }
     const int32_t unit_keys = choose_unit_keys(T, c.n_kv_heads, ctx->n_sm);
-    int32_t nu = 0;
+    int32_t nu = 0, nch = 0;
     int64_t list_off = 0, bound = 0;
     for (int r = 0; r < n_req; ++r) {
       ReqInfo& q = ctx->h_req[r];
@@ -217,9 +241,14 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
       q.N = (int32_t)(cu[r + 1] - cu[r]);
       q.n = q.N - c.window;
       q.keep_all = q.N <= c.total_budget / c.n_layers ? 1 : 0;
-      q.cap = (int32_t)(ctx->sel_budget < q.n ? ctx->sel_budget : q.n);
       q.list_off = list_off;
-      list_off += (int64_t)q.cap * c.n_layers * c.n_kv_heads;
+      list_off += (int64_t)q.n * c.n_layers * c.n_kv_heads;
+      q.nchunks = 0;
+      for (int32_t k0 = 0; k0 < q.N; k0 += kChunkKeys) {
+        ScoreUnit& u = ctx->h_chunks[nch++];
+        u.req = r; u.key0 = k0; u.nkeys = q.N - k0 < kChunkKeys ? q.N - k0 : kChunkKeys; u.pad = 0;
+        ++q.nchunks;
+      }
       q.unit0 = nu;
       for (int32_t k0 = 0; k0 < q.N; k0 += unit_keys) {
         ScoreUnit& u = ctx->h_units[nu++];
@@ -229,7 +258,8 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
       const int64_t full = (int64_t)c.n_layers * q.N;
       bound += (int64_t)c.n_kv_heads * (c.total_budget < full ? c.total_budget : full);
     }
-    if (list_off > ctx->list_elems || nu > ctx->max_units) return CAKE_ERR_CAPACITY;
+    if (list_off > ctx->list_elems || nu > ctx->max_units || nch > ctx->max_chunks) return CAKE_ERR_CAPACITY;
+    ctx->n_chunks = nch;
     if (ctx->use_tc) {
       const int32_t prc = tc_build_plan(ctx, n_req);
       if (prc != CAKE_OK) return prc;
@@ -240,6 +270,8 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
     CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_req, ctx->h_req, sizeof(ReqInfo) * n_req,
                                   cudaMemcpyHostToDevice, st));
     CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_units, ctx->h_units, sizeof(ScoreUnit) * nu,
+                                  cudaMemcpyHostToDevice, st));
+    CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_chunks, ctx->h_chunks, sizeof(ScoreUnit) * nch,
                                   cudaMemcpyHostToDevice, st));
     if (ctx->use_tc && ctx->n_tc_ctas > 0) {
       const size_t n_index = 2 * (size_t)(n_req * c.n_kv_heads + 1) + 2 * (size_t)(ctx->n_sm + 1);
@@ -252,7 +284,7 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
     CAKE_CUDA_TRY(cudaEventRecord(ctx->upload_done, st));
     ctx->upload_pending = true;
   }
-  if (n_req == 0) { ctx->n_units = 0; ctx->packed_rows_bound = 0; ctx->n_tc_ctas = 0; }
+  if (n_req == 0) { ctx->n_units = 0; ctx->n_chunks = 0; ctx->packed_rows_bound = 0; ctx->n_tc_ctas = 0; }
   if (ctx->use_tc) {
     ctx->tc_epoch = 0;
     CAKE_CUDA_TRY(cudaMemsetAsync(ctx->d_tc_sync, 0, sizeof(uint32_t) * 2 * ctx->max_pairs, st));
@@ -279,7 +311,7 @@ int32_t cake_score_layer(cake_ctx* ctx, int32_t layer, const void* q_win, const 
   const int sp = prof_begin(ctx, CAKE_PROF_FINALIZE, st);
   rc = launch_finalize_layer(ctx, layer, st);
   if (rc != CAKE_OK) return rc;
-  rc = launch_pool(ctx, st);
+  rc = launch_pool(ctx, layer, true, st);
   prof_end(ctx, sp, st);
   if (rc != CAKE_OK) return rc;
   ctx->n_ind = layer + 1;
@@ -376,6 +408,9 @@ int32_t cake_set_indicators(cake_ctx* ctx, int32_t layer, const float* in, void*
     CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_fresh, in,
                                   sizeof(float) * ctx->cfg.n_kv_heads * ctx->total_tokens,
                                   cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  // bucket histogram of the supplied values (they are taken as already pooled)
+  const int32_t rc = launch_pool(ctx, layer, false, (cudaStream_t)stream);
+  if (rc != CAKE_OK) return rc;
   ctx->n_ind = layer + 1;
   return CAKE_OK;
 }

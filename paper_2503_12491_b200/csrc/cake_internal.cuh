@@ -12,6 +12,10 @@ namespace cake {
 constexpr int kMaxRows = 128;        // G * S_w rows handled per KV head
 constexpr int kSimtTileKeys = 64;    // keys per tile of the SIMT score kernels
 constexpr int kSimtThreads = 256;
+constexpr int kBinBits = 12;         // survivor lists are sorted by the top bits of the indicator
+constexpr int kBins = 1 << kBinBits;
+constexpr int kChunkKeys = 4096;     // tokens per CTA of the pooling / scatter kernels
+constexpr int kBitmapSmemWords = 48 * 1024;   // positions of up to 1.5 M tokens are ordered in shared memory
 constexpr int kScoreGroups = 3;      // statistics warp groups per CTA of the tensor-core score kernel
 constexpr int kScoreWarps = 4 * kScoreGroups;   // statistics warps: one column-pass partial each
 
@@ -21,8 +25,8 @@ struct ReqInfo {
   int32_t N;         // prompt length
   int32_t n;         // N - S_w non-window tokens
   int32_t keep_all;  // 1: N <= floor(B_total/L), nothing is evicted
-  int32_t cap;       // capacity of each (layer, head) list = min(B', n)
-  int64_t list_off;  // first element of this request's lists in list_vals / list_pos
+  int32_t nchunks;   // chunks of kChunkKeys tokens covering the prompt
+  int64_t list_off;  // first entry of this request's lists; list (layer, head) holds n entries
   int32_t unit0;     // first score unit of the request
   int32_t nunits;    // number of score units of the request
 };
@@ -49,6 +53,15 @@ struct ScoreOp {
   int32_t seg;
   int32_t n;       // non-window keys of the request
   int32_t pad;
+};
+
+// Retained set of one (request, layer, head) list, whose entries (ordered key, position) are
+// stored by bucket.
+struct ListState {
+  int32_t bucket;        // threshold bucket d; all buckets before it are kept; -1: nothing kept
+  uint32_t thr_key;      // inside bucket d an entry is kept if key > thr_key,
+  int32_t pos_cut;       //   or key == thr_key and position <= pos_cut
+  int32_t kept;          // number of retained non-window tokens
 };
 
 struct LayerPtrs {
@@ -101,9 +114,21 @@ struct cake_ctx {
   int32_t* d_status;       // sticky device status word
   float* d_raw;            // [H_kv][max_total_tokens] un-pooled indicator
   float* d_fresh;          // [H_kv][max_total_tokens] pooled indicator of the newest layer
-  float* list_vals;        // per (req, layer, head) surviving indicators
-  int32_t* list_pos;       //                        and their token positions
+  uint2* d_lists;          // per (req, layer, head): n entries (ordered indicator key, position)
   int64_t list_elems;
+  int32_t* d_prefix;       // [max_lists][kBins+1] bucket offsets of every list
+  cake::ListState* d_lstate;   // [max_lists]
+  int64_t max_lists;
+  uint32_t* d_hist;        // [max_pairs][kBins] bucket histogram of the arriving layer (zero at rest)
+  uint32_t* d_fill;        // [max_pairs][kBins] scatter cursors (zero at rest)
+  uint32_t* d_arrivals;    // [max_pairs] chunk counters (zero at rest)
+  cake::ScoreUnit* h_chunks;   // pinned
+  cake::ScoreUnit* d_chunks;
+  int32_t n_chunks, max_chunks;
+  int32_t* d_pos_packed;   // [packed rows bound] positions in packed row order
+  int64_t pos_packed_cap;
+  uint32_t* d_bitmap;      // global bitmaps for requests too long for shared memory (or null)
+  int64_t bitmap_words;
   float* d_lse2;           // [max_requests][H_q][S_w] base-2 log-sum-exp of window rows
   float2* d_rowpart;       // [max_units][H_kv][R] (max, sum) partials of phase A
   float* d_colpart;        // [max_units][H_kv][G][2] partial (sum p*log2 p, sum var) of phase B
@@ -142,7 +167,7 @@ int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const f
                         cudaStream_t st);
 // cascade.cu
 int32_t launch_finalize_layer(cake_ctx* ctx, int32_t layer, cudaStream_t st);
-int32_t launch_pool(cake_ctx* ctx, cudaStream_t st);
+int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, cudaStream_t st);
 int32_t launch_allocate(cake_ctx* ctx, int32_t stage, cudaStream_t st);
 int32_t launch_evict(cake_ctx* ctx, int32_t stage, cudaStream_t st);
 // compact.cu

@@ -1,5 +1,5 @@
 // Layer finalisation (preference, pooling), the device-side budget allocator and
-// the per-head top-k eviction of the cascade.
+// the per-head top-k eviction of the cascade on bucket-sorted survivor lists.
 #include "cake_internal.cuh"
 
 #include <math_constants.h>
@@ -102,40 +102,123 @@ __global__ void finalize_layer_tc(const float* __restrict__ colpart,
   }
 }
 
-// --------------------------------------------------------------------- pool
-// fresh[g][t] = pool(raw[g][.]) over the request's non-window tokens; window
-// slots get +inf (Section 4.3).
-__global__ void pool_indicators(const float* __restrict__ raw, float* __restrict__ fresh,
-                                const ReqInfo* __restrict__ reqs, int n_req, int64_t T, int kp,
-                                int mode) {
-  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= T) return;
-  const int g = blockIdx.y;
-  int lo = 0, hi = n_req - 1;                 // last request with cu <= t
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (reqs[mid].cu <= t) lo = mid; else hi = mid - 1;
+// --------------------------------------------------------------- pool + bins
+// Survivor lists are kept sorted by bucket, not by position.  A key's bucket is the top
+// kBinBits bits of its order-preserving integer image, counted from the top (bucket 0 holds
+// the largest values).  When a layer arrives, its pooled indicators are histogrammed here and
+// scattered into bucket order by the eviction kernel; from then on "keep the top b" means
+// "all buckets before the one that contains the b-th element, plus the best part of that
+// bucket", so a later, smaller budget only moves a threshold and rewrites nothing.
+__device__ inline uint32_t ordered_key(float v) {
+  const uint32_t b = __float_as_uint(v);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ inline int bucket_of(uint32_t key) { return (kBins - 1) - (int)(key >> (32 - kBinBits)); }
+
+// Exclusive block scan (blockDim.x <= 1024) of one int per thread; *total gets the sum.
+__device__ inline int block_excl_scan(int v, int* warp_tot, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += n;
   }
-  const ReqInfo rq = reqs[lo];
-  const int j = (int)(t - rq.cu);
-  float out;
-  if (j >= rq.n) {
-    out = CUDART_INF_F;
-  } else {
-    const float* src = raw + (size_t)g * T + rq.cu;
-    const int r = kp >> 1;
-    const int a = max(0, j - r), b = min(rq.n, j + r + 1);
-    if (mode == CAKE_POOL_MAX) {
-      float m = src[a];
-      for (int x = a + 1; x < b; ++x) m = fmaxf(m, src[x]);
-      out = m;
-    } else {
-      float s = 0.f;
-      for (int x = a; x < b; ++x) s += src[x];
-      out = s / (float)kp;
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    const int w = lane < nw ? warp_tot[lane] : 0;
+    int winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += n;
     }
+    warp_tot[lane] = winc - w;
+    if (lane == 31) *total = winc;
   }
-  fresh[(size_t)g * T + t] = out;
+  __syncthreads();
+  const int r = warp_tot[warp] + inc - v;
+  __syncthreads();
+  return r;
+}
+
+constexpr int PH_THREADS = 256;
+
+// One CTA per (chunk of kChunkKeys tokens, KV head).  fresh[g][t] = pool(raw[g][.]) over the
+// request's non-window tokens, +inf on the window (Section 4.3); with do_pool = 0 the pooled
+// values are already in `fresh`.  The bucket histogram of the (request, head) is accumulated
+// in `hist`; the CTA that adds the last chunk turns it into the list's bucket offsets.
+__global__ void __launch_bounds__(PH_THREADS)
+pool_hist(const float* __restrict__ raw, float* __restrict__ fresh, const ReqInfo* __restrict__ reqs,
+          const ScoreUnit* __restrict__ chunks, uint32_t* __restrict__ hist,
+          uint32_t* __restrict__ arrivals, int32_t* __restrict__ prefix, int layer, int L, int Hkv,
+          int64_t T, int kp, int mode, int do_pool) {
+  __shared__ uint32_t sh[kBins];
+  __shared__ int warp_tot[32];
+  __shared__ int s_total, s_last;
+  const ScoreUnit ch = chunks[blockIdx.x];
+  const int g = blockIdx.y;
+  const ReqInfo rq = reqs[ch.req];
+  const int pair = ch.req * Hkv + g;
+  for (int b = threadIdx.x; b < kBins; b += PH_THREADS) sh[b] = 0;
+  __syncthreads();
+  const float* src = raw + (size_t)g * T + rq.cu;
+  float* dst = fresh + (size_t)g * T + rq.cu;
+  for (int i = threadIdx.x; i < ch.nkeys; i += PH_THREADS) {
+    const int j = ch.key0 + i;
+    float out;
+    if (j >= rq.n) {
+      out = CUDART_INF_F;
+    } else if (!do_pool) {
+      out = dst[j];
+    } else {
+      const int r = kp >> 1;
+      const int a = max(0, j - r), b = min(rq.n, j + r + 1);
+      if (mode == CAKE_POOL_MAX) {
+        float m = src[a];
+        for (int x = a + 1; x < b; ++x) m = fmaxf(m, src[x]);
+        out = m;
+      } else {
+        float s = 0.f;
+        for (int x = a; x < b; ++x) s += src[x];
+        out = s / (float)kp;
+      }
+    }
+    if (do_pool || j >= rq.n) dst[j] = out;
+    if (j < rq.n) atomicAdd(&sh[bucket_of(ordered_key(out))], 1u);
+  }
+  __syncthreads();
+  uint32_t* gh = hist + (size_t)pair * kBins;
+  for (int b = threadIdx.x; b < kBins; b += PH_THREADS)
+    if (sh[b]) atomicAdd(&gh[b], sh[b]);
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t old = atomicAdd(&arrivals[pair], 1u);
+    s_last = (old + 1u == (uint32_t)rq.nchunks) ? 1 : 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // bucket offsets of the new list: prefix[i] = elements in buckets before i
+  int32_t* pf = prefix + (((size_t)ch.req * L + layer) * Hkv + g) * (kBins + 1);
+  constexpr int PER = kBins / PH_THREADS;
+  int cnt[PER], sum = 0;
+#pragma unroll
+  for (int e = 0; e < PER; ++e) {
+    cnt[e] = (int)__ldcg(&gh[threadIdx.x * PER + e]);
+    sum += cnt[e];
+  }
+  int run = block_excl_scan(sum, warp_tot, &s_total);
+#pragma unroll
+  for (int e = 0; e < PER; ++e) {
+    pf[threadIdx.x * PER + e] = run;
+    run += cnt[e];
+    gh[threadIdx.x * PER + e] = 0;              // ready for the next layer
+  }
+  if (threadIdx.x == PH_THREADS - 1) pf[kBins] = run;
+  if (threadIdx.x == 0) arrivals[pair] = 0;
 }
 
 // ----------------------------------------------------------------- allocate
@@ -305,144 +388,223 @@ __global__ void allocate_budgets(const double* __restrict__ dP, const ReqInfo* _
 }
 
 // -------------------------------------------------------------------- evict
-constexpr int EV_THREADS = 1024;
-constexpr int EV_ITEMS = 8;
+constexpr int EV_THREADS = 256;
+constexpr int kTieCap = 2048;
 
-__device__ inline uint32_t ordered_key(float v) {
-  const uint32_t b = __float_as_uint(v);
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
+struct EvictSmem {
+  uint32_t hist[1024];
+  int32_t ties[kTieCap];
+  int warp_tot[32];
+  int total;
+  uint32_t sel_digit, sel_rem, sel_cnt;
+  int32_t tie_count, pos_cut;
+};
 
-// Exclusive block scan of two counters packed as (hi: a, lo: b) in 64 bits.
-__device__ inline unsigned long long block_excl_scan(unsigned long long v, unsigned long long* warp_tot,
-                                                     unsigned long long* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  unsigned long long inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const unsigned long long n = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += n;
-  }
-  if (lane == 31) warp_tot[warp] = inc;
+// Among `cnt` entries (all in one bucket), finds the digit (10 bits at `shift`) that holds the
+// krem-th largest key among the entries whose bits above shift+10 equal `prefix_bits`.
+__device__ inline void radix_digit(const uint2* __restrict__ e, int cnt, uint32_t mask,
+                                   uint32_t prefix_bits, int shift, uint32_t krem, EvictSmem& S) {
+  for (int b = threadIdx.x; b < 1024; b += blockDim.x) S.hist[b] = 0;
   __syncthreads();
-  if (warp == 0) {
-    unsigned long long w = lane < EV_THREADS / 32 ? warp_tot[lane] : 0ull;
-    unsigned long long winc = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned long long n = __shfl_up_sync(0xffffffffu, winc, o);
-      if (lane >= o) winc += n;
+  for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+    const uint32_t key = __ldcg(&e[i]).x;
+    if ((key & mask) == prefix_bits) atomicAdd(&S.hist[(key >> shift) & 1023u], 1u);
+  }
+  __syncthreads();
+  // digits from the top: thread t owns digits 1023-4t .. 1020-4t
+  const int per = 1024 / blockDim.x;
+  int mine = 0;
+  for (int q = 0; q < per; ++q) mine += (int)S.hist[1023 - (threadIdx.x * per + q)];
+  int above = block_excl_scan(mine, S.warp_tot, &S.total);
+  for (int q = 0; q < per; ++q) {
+    const int dg = 1023 - (threadIdx.x * per + q);
+    const int h = (int)S.hist[dg];
+    if ((uint32_t)above < krem && (uint32_t)(above + h) >= krem) {
+      S.sel_digit = (uint32_t)dg;
+      S.sel_rem = krem - (uint32_t)above;
+      S.sel_cnt = (uint32_t)h;
     }
-    warp_tot[lane] = winc - w;                 // exclusive prefix of warp totals
-    if (lane == 31) *total = winc;
+    above += h;
   }
   __syncthreads();
-  return warp_tot[warp] + inc - v;
 }
 
-// One CTA per (KV head, layer <= stage, request).  The newest layer reads the
-// pooled indicators with implicit positions; older layers read their stored list
-// and are compacted in place (an output slot never lies behind its source).
-__global__ void __launch_bounds__(EV_THREADS)
-evict_layers(const float* __restrict__ fresh, float* __restrict__ list_vals,
-             int32_t* __restrict__ list_pos, const ReqInfo* __restrict__ reqs,
-             const int32_t* __restrict__ prev, const int32_t* __restrict__ cur, int stage, int L,
-             int Hkv, int64_t T) {
-  __shared__ uint32_t hist[256];
-  __shared__ uint32_t s_prefix, s_krem;
-  __shared__ unsigned long long warp_tot[32];
-  __shared__ unsigned long long s_total;
-  const int g = blockIdx.x, layer = blockIdx.y, req = blockIdx.z;
-  const ReqInfo rq = reqs[req];
-  const bool is_new = layer == stage;
-  const int count = is_new ? rq.n : prev[(size_t)req * L + layer];
-  int k = cur[(size_t)req * L + layer];
-  k = min(k, count);
-  const size_t lbase = rq.list_off + ((size_t)layer * Hkv + g) * rq.cap;
-  float* lv = list_vals + lbase;
-  int32_t* lp = list_pos + lbase;
-  const float* src = is_new ? fresh + (size_t)g * T + rq.cu : lv;
-  if (k <= 0) return;
-  if (k >= count) {
-    if (is_new)
-      for (int j = threadIdx.x; j < count; j += EV_THREADS) { lv[j] = src[j]; lp[j] = j; }
+// Moves the threshold of one list to the budget b: the retained set becomes the first b entries
+// in the order (indicator descending, position ascending)  (Section 4.2 EVICT, Eq. 12).
+__device__ void set_threshold(const int32_t* __restrict__ pf, const uint2* __restrict__ list, int b,
+                              ListState* __restrict__ out, EvictSmem& S) {
+  if (b <= 0) {
+    if (threadIdx.x == 0) *out = ListState{-1, 0xFFFFFFFFu, -1, 0};
     return;
   }
-  // ---- radix select of the k-th largest key, 8 bits per pass from the top
-  uint32_t prefix = 0, mask = 0, krem = (uint32_t)k;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int b = threadIdx.x; b < 256; b += EV_THREADS) hist[b] = 0;
-    __syncthreads();
-    for (int j = threadIdx.x; j < count; j += EV_THREADS) {
-      const uint32_t key = ordered_key(src[j]);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      uint32_t above = 0;
-      int dsel = 0;
-      for (int dg = 255; dg >= 0; --dg) {
-        const uint32_t h = hist[dg];
-        if (above + h >= krem) { dsel = dg; break; }
-        above += h;
-      }
-      s_prefix = prefix | ((uint32_t)dsel << shift);
-      s_krem = krem - above;
-    }
-    __syncthreads();
-    prefix = s_prefix;
-    krem = s_krem;
-    mask |= 255u << shift;
-    __syncthreads();
+  // threshold bucket d: first bucket with prefix[d+1] >= b
+  int less = 0;
+  for (int i = threadIdx.x; i < kBins; i += blockDim.x) less += __ldcg(&pf[i + 1]) < b ? 1 : 0;
+  block_excl_scan(less, S.warp_tot, &S.total);
+  const int d = S.total;
+  __syncthreads();
+  if (d >= kBins) {                                  // b exceeds the stored entries: keep all
+    if (threadIdx.x == 0) *out = ListState{kBins - 1, 0u, 0x7FFFFFFF, __ldcg(&pf[kBins])};
+    return;
   }
-  const uint32_t thr = prefix;           // key of the k-th largest element
-  const uint32_t need_eq = krem;         // how many elements equal to it are kept (first by position)
-  // ---- ordered compaction
-  uint32_t gt_base = 0, eq_base = 0;
-  for (int c0 = 0; c0 < count; c0 += EV_THREADS * EV_ITEMS) {
-    float v[EV_ITEMS];
-    int32_t p[EV_ITEMS];
-    uint32_t fl[EV_ITEMS];
-    uint32_t cg = 0, ce = 0;
-    const int j0 = c0 + threadIdx.x * EV_ITEMS;
-#pragma unroll
-    for (int e = 0; e < EV_ITEMS; ++e) {
-      const int j = j0 + e;
-      fl[e] = 0;
-      if (j < count) {
-        v[e] = src[j];
-        p[e] = is_new ? j : lp[j];
-        const uint32_t key = ordered_key(v[e]);
-        fl[e] = key > thr ? 1u : (key == thr ? 2u : 0u);
-        cg += fl[e] == 1u;
-        ce += fl[e] == 2u;
+  const int start = __ldcg(&pf[d]), cnt = __ldcg(&pf[d + 1]) - start;
+  const uint32_t rem = (uint32_t)(b - start);
+  if ((int)rem >= cnt) {
+    if (threadIdx.x == 0) *out = ListState{d, 0u, 0x7FFFFFFF, b};
+    return;
+  }
+  const uint2* e = list + start;
+  constexpr int low = 32 - kBinBits;                 // key bits below the bucket bits (20)
+  radix_digit(e, cnt, 0u, 0u, low - 10, rem, S);
+  uint32_t pre = S.sel_digit << (low - 10);
+  uint32_t krem = S.sel_rem;
+  __syncthreads();
+  radix_digit(e, cnt, 1023u << (low - 10), pre, 0, krem, S);
+  pre |= S.sel_digit;
+  const uint32_t need_eq = S.sel_rem, n_eq = S.sel_cnt;
+  __syncthreads();
+  // full key of the threshold: bucket bits + the 20 selected bits
+  const uint32_t thr = ((uint32_t)(kBins - 1 - d) << low) | pre;
+  int32_t pos_cut = 0x7FFFFFFF;
+  if (need_eq < n_eq) {
+    // ties at the threshold: the need_eq lowest positions win
+    if (threadIdx.x == 0) { S.tie_count = 0; S.pos_cut = 0x7FFFFFFF; }
+    __syncthreads();
+    if (n_eq <= (uint32_t)kTieCap) {
+      for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+        const uint2 v = __ldcg(&e[i]);
+        if (v.x == thr) S.ties[atomicAdd(&S.tie_count, 1)] = (int32_t)v.y;
       }
-    }
-    unsigned long long tot;
-    const unsigned long long ex =
-        block_excl_scan(((unsigned long long)cg << 32) | ce, warp_tot, &s_total);
-    tot = s_total;
-    uint32_t gt_before = gt_base + (uint32_t)(ex >> 32);
-    uint32_t eq_before = eq_base + (uint32_t)(ex & 0xffffffffu);
-    // all reads of this chunk are done (block_excl_scan synchronised) -> safe to write in place
-#pragma unroll
-    for (int e = 0; e < EV_ITEMS; ++e) {
-      if (fl[e] == 1u) {
-        const uint32_t o = gt_before + min(eq_before, need_eq);
-        lv[o] = v[e]; lp[o] = p[e];
-        ++gt_before;
-      } else if (fl[e] == 2u) {
-        if (eq_before < need_eq) {
-          const uint32_t o = gt_before + eq_before;
-          lv[o] = v[e]; lp[o] = p[e];
+      __syncthreads();
+      for (int i = threadIdx.x; i < (int)n_eq; i += blockDim.x) {
+        const int32_t p = S.ties[i];
+        uint32_t r = 0;
+        for (int o = 0; o < (int)n_eq; ++o) r += S.ties[o] < p ? 1u : 0u;
+        if (r == need_eq - 1) S.pos_cut = p;
+      }
+      __syncthreads();
+    } else {
+      // many ties: bisect the position (positions are distinct)
+      int lo = 0, hi = 0x7FFFFFFF;                   // smallest cut with count(pos <= cut) >= need_eq
+      while (lo < hi) {
+        const int mid = lo + ((hi - lo) >> 1);
+        int c = 0;
+        for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+          const uint2 v = __ldcg(&e[i]);
+          c += (v.x == thr && (int32_t)v.y <= mid) ? 1 : 0;
         }
-        ++eq_before;
+        block_excl_scan(c, S.warp_tot, &S.total);
+        const int tot = S.total;
+        __syncthreads();
+        if ((uint32_t)tot >= need_eq) hi = mid; else lo = mid + 1;
       }
+      if (threadIdx.x == 0) S.pos_cut = lo;
+      __syncthreads();
     }
-    gt_base += (uint32_t)(tot >> 32);
-    eq_base += (uint32_t)(tot & 0xffffffffu);
-    __syncthreads();
+    pos_cut = S.pos_cut;
   }
+  if (threadIdx.x == 0) *out = ListState{d, thr, pos_cut, b};
+}
+
+struct EvictArgs {
+  const float* fresh;
+  uint2* lists;
+  const int32_t* prefix_all;
+  ListState* states;
+  uint32_t* fill;          // [pairs][kBins], zero between launches
+  uint32_t* arrivals;      // [pairs]
+  const ReqInfo* reqs;
+  const ScoreUnit* chunks;
+  const int32_t* cur;      // budgets of this stage
+  int n_chunks, stage, L, Hkv, n_req;
+  int64_t T;
+};
+
+// Stage `stage` of the cascade.  CTAs [0, n_chunks * Hkv): scatter one chunk of the newest
+// layer's pooled indicators into bucket order (only the buckets its budget can ever reach; the
+// budget never grows again, Proposition 1); the CTA that completes a list sets its threshold.
+// The remaining CTAs move the threshold of one older list each to its new budget.
+__global__ void __launch_bounds__(EV_THREADS)
+evict_stage(const EvictArgs A) {
+  __shared__ EvictSmem S;
+  __shared__ uint32_t s_cnt[kBins];
+  __shared__ uint32_t s_base[kBins];
+  __shared__ int s_last;
+  const int n_scatter = A.n_chunks * A.Hkv;
+  if ((int)blockIdx.x >= n_scatter) {
+    // ---- older list: (request, layer < stage, head)
+    int idx = (int)blockIdx.x - n_scatter;
+    const int g = idx % A.Hkv; idx /= A.Hkv;
+    const int layer = idx % A.stage;
+    const int req = idx / A.stage;
+    const ReqInfo rq = A.reqs[req];
+    const size_t lid = ((size_t)req * A.L + layer) * A.Hkv + g;
+    const int b = min(A.cur[(size_t)req * A.L + layer], rq.n);
+    if (A.states[lid].kept == b) return;                       // budget unchanged
+    set_threshold(A.prefix_all + lid * (kBins + 1),
+                  A.lists + rq.list_off + ((size_t)layer * A.Hkv + g) * rq.n, b, &A.states[lid], S);
+    return;
+  }
+  // ---- newest layer: scatter chunk
+  const ScoreUnit ch = A.chunks[blockIdx.x / A.Hkv];
+  const int g = blockIdx.x % A.Hkv;
+  const ReqInfo rq = A.reqs[ch.req];
+  const int pair = ch.req * A.Hkv + g;
+  const size_t lid = ((size_t)ch.req * A.L + A.stage) * A.Hkv + g;
+  const int32_t* pf = A.prefix_all + lid * (kBins + 1);
+  uint2* list = A.lists + rq.list_off + ((size_t)A.stage * A.Hkv + g) * rq.n;
+  const int b = min(A.cur[(size_t)ch.req * A.L + A.stage], rq.n);
+  // last bucket worth storing
+  int less = 0;
+  for (int i = threadIdx.x; i < kBins; i += EV_THREADS) {
+    less += __ldcg(&pf[i + 1]) < b ? 1 : 0;
+    s_cnt[i] = 0;
+  }
+  block_excl_scan(less, S.warp_tot, &S.total);
+  const int d_last = b > 0 ? min(S.total, kBins - 1) : -1;
+  __syncthreads();
+  constexpr int PER = kChunkKeys / EV_THREADS;
+  uint32_t key[PER];
+  int bk[PER];
+  const float* src = A.fresh + (size_t)g * A.T + rq.cu;
+#pragma unroll
+  for (int e = 0; e < PER; ++e) {
+    const int i = threadIdx.x + e * EV_THREADS;
+    const int j = ch.key0 + i;
+    bk[e] = -1;
+    if (i < ch.nkeys && j < rq.n) {
+      key[e] = ordered_key(src[j]);
+      const int q = bucket_of(key[e]);
+      if (q <= d_last) { bk[e] = q; atomicAdd(&s_cnt[q], 1u); }
+    }
+  }
+  __syncthreads();
+  uint32_t* gf = A.fill + (size_t)pair * kBins;
+  for (int q = threadIdx.x; q < kBins; q += EV_THREADS) {
+    const uint32_t c = s_cnt[q];
+    if (c) s_base[q] = (uint32_t)__ldcg(&pf[q]) + atomicAdd(&gf[q], c);
+    s_cnt[q] = 0;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int e = 0; e < PER; ++e) {
+    if (bk[e] >= 0) {
+      const uint32_t off = s_base[bk[e]] + atomicAdd(&s_cnt[bk[e]], 1u);
+      list[off] = make_uint2(key[e], (uint32_t)(ch.key0 + threadIdx.x + e * EV_THREADS));
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t old = atomicAdd(&A.arrivals[pair], 1u);
+    s_last = (old + 1u == (uint32_t)rq.nchunks) ? 1 : 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int q = threadIdx.x; q < kBins; q += EV_THREADS) gf[q] = 0;       // ready for the next stage
+  if (threadIdx.x == 0) A.arrivals[pair] = 0;
+  set_threshold(pf, list, b, &A.states[lid], S);
 }
 
 }  // namespace
@@ -467,12 +629,14 @@ int32_t launch_finalize_layer(cake_ctx* ctx, int32_t layer, cudaStream_t st) {
   return cuda_status(cudaGetLastError());
 }
 
-int32_t launch_pool(cake_ctx* ctx, cudaStream_t st) {
+int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, cudaStream_t st) {
   const cake_config& c = ctx->cfg;
-  if (ctx->n_req == 0 || ctx->total_tokens == 0) return CAKE_OK;
-  const dim3 grid((unsigned)((ctx->total_tokens + 255) / 256), c.n_kv_heads);
-  pool_indicators<<<grid, 256, 0, st>>>(ctx->d_raw, ctx->d_fresh, ctx->d_req, ctx->n_req,
-                                        ctx->total_tokens, c.pool_kernel, c.pool_mode);
+  if (ctx->n_req == 0 || ctx->n_chunks == 0) return CAKE_OK;
+  const dim3 grid((unsigned)ctx->n_chunks, c.n_kv_heads);
+  pool_hist<<<grid, PH_THREADS, 0, st>>>(ctx->d_raw, ctx->d_fresh, ctx->d_req, ctx->d_chunks,
+                                         ctx->d_hist, ctx->d_arrivals, ctx->d_prefix, layer,
+                                         c.n_layers, c.n_kv_heads, ctx->total_tokens, c.pool_kernel,
+                                         c.pool_mode, do_pool ? 1 : 0);
   count_launch();
   return cuda_status(cudaGetLastError());
 }
@@ -490,10 +654,22 @@ int32_t launch_allocate(cake_ctx* ctx, int32_t stage, cudaStream_t st) {
 int32_t launch_evict(cake_ctx* ctx, int32_t stage, cudaStream_t st) {
   const cake_config& c = ctx->cfg;
   if (ctx->n_req == 0) return CAKE_OK;
-  const dim3 grid(c.n_kv_heads, stage + 1, ctx->n_req);
-  evict_layers<<<grid, EV_THREADS, 0, st>>>(ctx->d_fresh, ctx->list_vals, ctx->list_pos, ctx->d_req,
-                                            ctx->d_budget[(stage + 1) & 1], ctx->d_budget[stage & 1],
-                                            stage, c.n_layers, c.n_kv_heads, ctx->total_tokens);
+  EvictArgs A;
+  A.fresh = ctx->d_fresh;
+  A.lists = ctx->d_lists;
+  A.prefix_all = ctx->d_prefix;
+  A.states = ctx->d_lstate;
+  A.fill = ctx->d_fill;
+  A.arrivals = ctx->d_arrivals;
+  A.reqs = ctx->d_req;
+  A.chunks = ctx->d_chunks;
+  A.cur = ctx->d_budget[stage & 1];
+  A.n_chunks = ctx->n_chunks; A.stage = stage; A.L = c.n_layers; A.Hkv = c.n_kv_heads;
+  A.n_req = ctx->n_req;
+  A.T = ctx->total_tokens;
+  const unsigned grid = (unsigned)(ctx->n_chunks * c.n_kv_heads + stage * c.n_kv_heads * ctx->n_req);
+  if (grid == 0) return CAKE_OK;
+  evict_stage<<<grid, EV_THREADS, 0, st>>>(A);
   count_launch();
   return cuda_status(cudaGetLastError());
 }
