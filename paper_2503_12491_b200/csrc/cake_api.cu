@@ -61,7 +61,7 @@ void free_ctx(cake_ctx* c) {
   cudaFree(c->d_req); cudaFree(c->d_units); cudaFree(c->d_H); cudaFree(c->d_V); cudaFree(c->d_P);
   cudaFree(c->d_budget[0]); cudaFree(c->d_budget[1]); cudaFree(c->d_status); cudaFree(c->d_raw);
   cudaFree(c->d_fresh); cudaFree(c->d_lists); cudaFree(c->d_prefix); cudaFree(c->d_lstate);
-  cudaFree(c->d_hist); cudaFree(c->d_fill); cudaFree(c->d_arrivals); cudaFree(c->d_chunks);
+  cudaFree(c->d_hist); cudaFree(c->d_fill); cudaFree(c->d_arrivals); cudaFree(c->d_headsum); cudaFree(c->d_chunks);
   cudaFree(c->d_pos_packed); cudaFree(c->d_bitmap); cudaFree(c->d_lse2);
   if (c->h_chunks) cudaFreeHost(c->h_chunks);
   cudaFree(c->d_rowpart); cudaFree(c->d_colpart);
@@ -157,14 +157,15 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   ok = ok && dev_alloc(&x->d_lstate, (size_t)x->max_lists) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_hist, (size_t)R * c.n_kv_heads * kBins) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_fill, (size_t)R * c.n_kv_heads * kBins) == cudaSuccess;
-  ok = ok && dev_alloc(&x->d_arrivals, (size_t)R * c.n_kv_heads) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_arrivals, (size_t)R * c.n_kv_heads + R) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_headsum, (size_t)R * c.n_q_heads * 2) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_chunks, (size_t)x->max_chunks) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_pos_packed, (size_t)x->pos_packed_cap) == cudaSuccess;
   if (x->bitmap_words > 0) ok = ok && dev_alloc(&x->d_bitmap, (size_t)x->bitmap_words) == cudaSuccess;
   ok = ok && cudaMallocHost((void**)&x->h_chunks, sizeof(ScoreUnit) * x->max_chunks) == cudaSuccess;
   ok = ok && cudaMemset(x->d_hist, 0, sizeof(uint32_t) * R * c.n_kv_heads * kBins) == cudaSuccess;
   ok = ok && cudaMemset(x->d_fill, 0, sizeof(uint32_t) * R * c.n_kv_heads * kBins) == cudaSuccess;
-  ok = ok && cudaMemset(x->d_arrivals, 0, sizeof(uint32_t) * R * c.n_kv_heads) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_arrivals, 0, sizeof(uint32_t) * (R * c.n_kv_heads + R)) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_lse2, (size_t)R * c.n_q_heads * c.window) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_rowpart, (size_t)x->max_units * c.n_kv_heads * x->rows) == cudaSuccess;
   {
@@ -309,9 +310,7 @@ int32_t cake_score_layer(cake_ctx* ctx, int32_t layer, const void* q_win, const 
                            : launch_score_simt(ctx, q_win, k, lse, st);
   if (rc != CAKE_OK) return rc;
   const int sp = prof_begin(ctx, CAKE_PROF_FINALIZE, st);
-  rc = launch_finalize_layer(ctx, layer, st);
-  if (rc != CAKE_OK) return rc;
-  rc = launch_pool(ctx, layer, true, st);
+  rc = launch_pool(ctx, layer, true, true, st);
   prof_end(ctx, sp, st);
   if (rc != CAKE_OK) return rc;
   ctx->n_ind = layer + 1;
@@ -409,7 +408,7 @@ int32_t cake_set_indicators(cake_ctx* ctx, int32_t layer, const float* in, void*
                                   sizeof(float) * ctx->cfg.n_kv_heads * ctx->total_tokens,
                                   cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
   // bucket histogram of the supplied values (they are taken as already pooled)
-  const int32_t rc = launch_pool(ctx, layer, false, (cudaStream_t)stream);
+  const int32_t rc = launch_pool(ctx, layer, false, false, (cudaStream_t)stream);
   if (rc != CAKE_OK) return rc;
   ctx->n_ind = layer + 1;
   return CAKE_OK;

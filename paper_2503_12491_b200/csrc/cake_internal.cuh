@@ -121,7 +121,8 @@ struct cake_ctx {
   int64_t max_lists;
   uint32_t* d_hist;        // [max_pairs][kBins] bucket histogram of the arriving layer (zero at rest)
   uint32_t* d_fill;        // [max_pairs][kBins] scatter cursors (zero at rest)
-  uint32_t* d_arrivals;    // [max_pairs] chunk counters (zero at rest)
+  uint32_t* d_arrivals;    // [max_pairs] chunk counters, then [max_requests] head counters (zero at rest)
+  double* d_headsum;       // [max_requests][H_q][2] per-head entropy / variance sums of the layer
   cake::ScoreUnit* h_chunks;   // pinned
   cake::ScoreUnit* d_chunks;
   int32_t n_chunks, max_chunks;
@@ -166,8 +167,7 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req);
 int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const float* lse,
                         cudaStream_t st);
 // cascade.cu
-int32_t launch_finalize_layer(cake_ctx* ctx, int32_t layer, cudaStream_t st);
-int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, cudaStream_t st);
+int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, bool finalize, cudaStream_t st);
 int32_t launch_allocate(cake_ctx* ctx, int32_t stage, cudaStream_t st);
 int32_t launch_evict(cake_ctx* ctx, int32_t stage, cudaStream_t st);
 // compact.cu

@@ -4,6 +4,8 @@
 
 #include <math_constants.h>
 
+#include <cstring>
+
 namespace cake {
 namespace {
 
@@ -59,49 +61,6 @@ __device__ inline double warp_sum_f64(double v) {
   return v;
 }
 
-__global__ void finalize_layer_tc(const float* __restrict__ colpart,
-                                  const int32_t* __restrict__ pair_seg,
-                                  const float* __restrict__ hrow, int use_hrow, int rows,
-                                  double* __restrict__ dH, double* __restrict__ dV,
-                                  double* __restrict__ dP, int32_t* __restrict__ status, int layer,
-                                  int L, int Hq, int Hkv, double inv_tau1, double inv_tau2) {
-  __shared__ double sh[2][32];
-  const int req = blockIdx.x;
-  const int G = Hq / Hkv;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
-  double hsum = 0.0, vsum = 0.0;                         // per warp, over its heads
-  for (int h = warp; h < Hq; h += nwarp) {
-    const int g = h / G, hl = h - g * G;
-    const int pair = req * Hkv + g;
-    double a = 0.0, b = 0.0;
-    const int s_lo = pair_seg[pair] * kScoreWarps, s_hi = pair_seg[pair + 1] * kScoreWarps;
-    for (int sg = s_lo + lane; sg < s_hi; sg += 32) {
-      const float2 p = *reinterpret_cast<const float2*>(colpart + ((size_t)sg * G + hl) * 2);
-      a += (double)p.x;
-      b += (double)p.y;
-    }
-    if (use_hrow) {
-      a = 0.0;
-      for (int r = hl + lane * G; r < rows; r += 32 * G) a += (double)hrow[(size_t)pair * 128 + r];
-    }
-    hsum += -0.6931471805599453 * warp_sum_f64(a);
-    vsum += warp_sum_f64(b);
-  }
-  if (lane == 0) { sh[0][warp] = hsum; sh[1][warp] = vsum; }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double H = 0.0, V = 0.0;
-    for (int t = 0; t < nwarp; ++t) { H += sh[0][t]; V += sh[1][t]; }
-    H /= (double)Hq;
-    V /= (double)Hq;
-    const double P = pow(H, inv_tau1) * pow(V, inv_tau2);
-    dH[(size_t)req * L + layer] = H;
-    dV[(size_t)req * L + layer] = V;
-    dP[(size_t)req * L + layer] = P;
-    if (!(P >= 0.0) || isinf(P)) raise_status(status, CAKE_ERR_NONFINITE);
-  }
-}
-
 // --------------------------------------------------------------- pool + bins
 // Survivor lists are kept sorted by bucket, not by position.  A key's bucket is the top
 // kBinBits bits of its order-preserving integer image, counted from the top (bucket 0 holds
@@ -144,16 +103,91 @@ __device__ inline int block_excl_scan(int v, int* warp_tot, int* total) {
 }
 
 constexpr int PH_THREADS = 256;
+constexpr int PH_PER = kChunkKeys / PH_THREADS;      // consecutive tokens per thread
 
-// One CTA per (chunk of kChunkKeys tokens, KV head).  fresh[g][t] = pool(raw[g][.]) over the
-// request's non-window tokens, +inf on the window (Section 4.3); with do_pool = 0 the pooled
-// values are already in `fresh`.  The bucket histogram of the (request, head) is accumulated
-// in `hist`; the CTA that adds the last chunk turns it into the list's bucket offsets.
+struct FinalizeArgs {        // preference of the layer from the tensor-core kernel's partials
+  const float* colpart;      // [pass-B segment][statistics warp][G][2]
+  const int32_t* pair_seg;   // [pairs + 1]
+  const float* hrow;         // [pair][128] or unused
+  double* headsum;           // [req][H_q][2] scratch
+  uint32_t* fin_arrivals;    // [req], zero at rest
+  double* dH; double* dV; double* dP;
+  int32_t* status;
+  int units;                 // extra CTAs per KV head: n_req * G (0 = none)
+  int use_hrow, rows, Hq;
+  double inv_tau1, inv_tau2;
+};
+
+// H_h = -ln2 * sum p*log2(p), V_h = sum_j Var_i of one query head; the CTA that finishes a
+// request's last head averages over the heads and sets P = H^(1/tau1) * V^(1/tau2) (Eq. 4-6).
+// All sums run in a fixed order in double precision.
+__device__ void finalize_head(const FinalizeArgs& F, int req, int g, int hl, int layer, int L, int Hkv) {
+  __shared__ double red[2][PH_THREADS / 32];
+  __shared__ int s_last;
+  const int G = F.Hq / Hkv;
+  const int pair = req * Hkv + g;
+  double a = 0.0, b = 0.0;
+  const int s_lo = F.pair_seg[pair] * kScoreWarps, s_hi = F.pair_seg[pair + 1] * kScoreWarps;
+  for (int sg = s_lo + (int)threadIdx.x; sg < s_hi; sg += PH_THREADS) {
+    const float2 p = __ldcg(reinterpret_cast<const float2*>(F.colpart + ((size_t)sg * G + hl) * 2));
+    a += (double)p.x;
+    b += (double)p.y;
+  }
+  if (F.use_hrow) {
+    a = 0.0;
+    for (int r = hl + (int)threadIdx.x * G; r < F.rows; r += PH_THREADS * G)
+      a += (double)__ldcg(&F.hrow[(size_t)pair * 128 + r]);
+  }
+  a = warp_sum_f64(a);
+  b = warp_sum_f64(b);
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = a; red[1][threadIdx.x >> 5] = b; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double ha = 0.0, vb = 0.0;
+    for (int w = 0; w < PH_THREADS / 32; ++w) { ha += red[0][w]; vb += red[1][w]; }
+    double* hs = F.headsum + ((size_t)req * F.Hq + g * G + hl) * 2;
+    hs[0] = -0.6931471805599453 * ha;
+    hs[1] = vb;
+    __threadfence();
+    const uint32_t old = atomicAdd(&F.fin_arrivals[req], 1u);
+    s_last = (old + 1u == (uint32_t)F.Hq) ? 1 : 0;
+    if (s_last) {
+      __threadfence();
+      F.fin_arrivals[req] = 0;
+      double H = 0.0, V = 0.0;
+      for (int h = 0; h < F.Hq; ++h) {
+        H += __ldcg(&F.headsum[((size_t)req * F.Hq + h) * 2]);
+        V += __ldcg(&F.headsum[((size_t)req * F.Hq + h) * 2 + 1]);
+      }
+      H /= (double)F.Hq;
+      V /= (double)F.Hq;
+      const double P = pow(H, F.inv_tau1) * pow(V, F.inv_tau2);
+      F.dH[(size_t)req * L + layer] = H;
+      F.dV[(size_t)req * L + layer] = V;
+      F.dP[(size_t)req * L + layer] = P;
+      if (!(P >= 0.0) || isinf(P)) raise_status(F.status, CAKE_ERR_NONFINITE);
+    }
+  }
+}
+
+// One CTA per (chunk of kChunkKeys tokens, KV head); a thread owns PH_PER consecutive tokens.
+// fresh[g][t] = pool(raw[g][.]) over the request's non-window tokens, +inf on the window
+// (Section 4.3); with do_pool = 0 the pooled values are already in `fresh`.  The bucket
+// histogram of the (request, head) is accumulated in `hist`; the CTA that adds the last chunk
+// turns it into the list's bucket offsets.  R = pool_kernel / 2 when that is at most 3, else
+// -1 (any kernel size, one global read per tap).  CTAs past the chunks finalise the layer's
+// preference (tensor-core path).
+template <int R>
 __global__ void __launch_bounds__(PH_THREADS)
 pool_hist(const float* __restrict__ raw, float* __restrict__ fresh, const ReqInfo* __restrict__ reqs,
           const ScoreUnit* __restrict__ chunks, uint32_t* __restrict__ hist,
-          uint32_t* __restrict__ arrivals, int32_t* __restrict__ prefix, int layer, int L, int Hkv,
-          int64_t T, int kp, int mode, int do_pool) {
+          uint32_t* __restrict__ arrivals, int32_t* __restrict__ prefix, int n_chunks, int layer,
+          int L, int Hkv, int64_t T, int kp, int mode, int do_pool, const FinalizeArgs F) {
+  if ((int)blockIdx.x >= n_chunks) {
+    const int ex = (int)blockIdx.x - n_chunks, G = F.Hq / Hkv;
+    finalize_head(F, ex / G, blockIdx.y, ex % G, layer, L, Hkv);
+    return;
+  }
   __shared__ uint32_t sh[kBins];
   __shared__ int warp_tot[32];
   __shared__ int s_total, s_last;
@@ -165,29 +199,63 @@ pool_hist(const float* __restrict__ raw, float* __restrict__ fresh, const ReqInf
   __syncthreads();
   const float* src = raw + (size_t)g * T + rq.cu;
   float* dst = fresh + (size_t)g * T + rq.cu;
-  for (int i = threadIdx.x; i < ch.nkeys; i += PH_THREADS) {
-    const int j = ch.key0 + i;
-    float out;
-    if (j >= rq.n) {
-      out = CUDART_INF_F;
-    } else if (!do_pool) {
-      out = dst[j];
-    } else {
-      const int r = kp >> 1;
-      const int a = max(0, j - r), b = min(rq.n, j + r + 1);
-      if (mode == CAKE_POOL_MAX) {
-        float m = src[a];
-        for (int x = a + 1; x < b; ++x) m = fmaxf(m, src[x]);
-        out = m;
+  const int j0 = ch.key0 + (int)threadIdx.x * PH_PER;
+  float out[PH_PER];
+  if (!do_pool) {
+#pragma unroll
+    for (int e = 0; e < PH_PER; ++e) out[e] = j0 + e < rq.n ? dst[j0 + e] : CUDART_INF_F;
+  } else if (R >= 0) {
+    const float pad = mode == CAKE_POOL_MAX ? -CUDART_INF_F : 0.f;
+    float w[PH_PER + 2 * (R >= 0 ? R : 0)];
+#pragma unroll
+    for (int x = 0; x < PH_PER + 2 * R; ++x) {
+      const int j = j0 - R + x;
+      w[x] = (j >= 0 && j < rq.n) ? src[j] : pad;
+    }
+#pragma unroll
+    for (int e = 0; e < PH_PER; ++e) {
+      float m = w[e];
+#pragma unroll
+      for (int x = 1; x <= 2 * R; ++x) m = mode == CAKE_POOL_MAX ? fmaxf(m, w[e + x]) : m + w[e + x];
+      out[e] = mode == CAKE_POOL_MAX ? m : m / (float)kp;
+    }
+  } else {
+    const int r = kp >> 1;
+#pragma unroll 1
+    for (int e = 0; e < PH_PER; ++e) {
+      const int j = j0 + e;
+      float m = 0.f;
+      if (j < rq.n) {
+        const int a = max(0, j - r), b = min(rq.n, j + r + 1);
+        m = src[a];
+        for (int x = a + 1; x < b; ++x) m = mode == CAKE_POOL_MAX ? fmaxf(m, src[x]) : m + src[x];
+        if (mode != CAKE_POOL_MAX) m /= (float)kp;
+      }
+      out[e] = m;
+    }
+  }
+  // write back and count buckets; neighbours often share a bucket, so runs are counted once
+  int run_bin = -1;
+  uint32_t run_len = 0;
+#pragma unroll
+  for (int e = 0; e < PH_PER; ++e) {
+    const int j = j0 + e;
+    if (j < ch.key0 + ch.nkeys) {
+      if (j >= rq.n) {
+        dst[j] = CUDART_INF_F;
       } else {
-        float s = 0.f;
-        for (int x = a; x < b; ++x) s += src[x];
-        out = s / (float)kp;
+        if (do_pool) dst[j] = out[e];
+        const int q = bucket_of(ordered_key(out[e]));
+        if (q != run_bin) {
+          if (run_len) atomicAdd(&sh[run_bin], run_len);
+          run_bin = q;
+          run_len = 0;
+        }
+        ++run_len;
       }
     }
-    if (do_pool || j >= rq.n) dst[j] = out;
-    if (j < rq.n) atomicAdd(&sh[bucket_of(ordered_key(out))], 1u);
   }
+  if (run_len) atomicAdd(&sh[run_bin], run_len);
   __syncthreads();
   uint32_t* gh = hist + (size_t)pair * kBins;
   for (int b = threadIdx.x; b < kBins; b += PH_THREADS)
@@ -563,20 +631,35 @@ evict_stage(const EvictArgs A) {
   block_excl_scan(less, S.warp_tot, &S.total);
   const int d_last = b > 0 ? min(S.total, kBins - 1) : -1;
   __syncthreads();
+  // a thread owns PER consecutive tokens; runs of equal buckets are counted and placed at once
   constexpr int PER = kChunkKeys / EV_THREADS;
   uint32_t key[PER];
   int bk[PER];
   const float* src = A.fresh + (size_t)g * A.T + rq.cu;
+  const int j0 = ch.key0 + (int)threadIdx.x * PER;
 #pragma unroll
   for (int e = 0; e < PER; ++e) {
-    const int i = threadIdx.x + e * EV_THREADS;
-    const int j = ch.key0 + i;
+    const int j = j0 + e;
     bk[e] = -1;
-    if (i < ch.nkeys && j < rq.n) {
+    if (j < rq.n && j < ch.key0 + ch.nkeys) {
       key[e] = ordered_key(src[j]);
       const int q = bucket_of(key[e]);
-      if (q <= d_last) { bk[e] = q; atomicAdd(&s_cnt[q], 1u); }
+      if (q <= d_last) bk[e] = q;
     }
+  }
+  {
+    int run_bin = -1;
+    uint32_t run_len = 0;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) {
+      if (bk[e] != run_bin) {
+        if (run_len && run_bin >= 0) atomicAdd(&s_cnt[run_bin], run_len);
+        run_bin = bk[e];
+        run_len = 0;
+      }
+      ++run_len;
+    }
+    if (run_len && run_bin >= 0) atomicAdd(&s_cnt[run_bin], run_len);
   }
   __syncthreads();
   uint32_t* gf = A.fill + (size_t)pair * kBins;
@@ -586,11 +669,24 @@ evict_stage(const EvictArgs A) {
     s_cnt[q] = 0;
   }
   __syncthreads();
+  {
+    int run_bin = -1;
+    uint32_t run_off = 0;
 #pragma unroll
-  for (int e = 0; e < PER; ++e) {
-    if (bk[e] >= 0) {
-      const uint32_t off = s_base[bk[e]] + atomicAdd(&s_cnt[bk[e]], 1u);
-      list[off] = make_uint2(key[e], (uint32_t)(ch.key0 + threadIdx.x + e * EV_THREADS));
+    for (int e = 0; e < PER; ++e) {
+      if (bk[e] != run_bin) {
+        run_bin = bk[e];
+        if (run_bin >= 0) {
+          uint32_t len = 1;
+#pragma unroll
+          for (int f = e + 1; f < PER; ++f) {
+            if (bk[f] != run_bin) break;
+            ++len;
+          }
+          run_off = s_base[run_bin] + atomicAdd(&s_cnt[run_bin], len);
+        }
+      }
+      if (run_bin >= 0) list[run_off++] = make_uint2(key[e], (uint32_t)(j0 + e));
     }
   }
   __threadfence();
@@ -609,34 +705,52 @@ evict_stage(const EvictArgs A) {
 
 }  // namespace
 
-int32_t launch_finalize_layer(cake_ctx* ctx, int32_t layer, cudaStream_t st) {
+// Pooling + bucket histogram of layer `layer`; with `finalize` also the layer's preference
+// (tensor-core path: extra CTAs of the same launch; SIMT path: its own small kernel).
+int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, bool finalize, cudaStream_t st) {
   const cake_config& c = ctx->cfg;
   if (ctx->n_req == 0) return CAKE_OK;
-  if (ctx->use_tc) {
-    finalize_layer_tc<<<ctx->n_req, 1024, 0, st>>>(
-        ctx->d_colpart, ctx->d_tc_index + (ctx->n_req * c.n_kv_heads + 1), ctx->d_hrow,
-        ctx->hhead_from_rows ? 1 : 0, ctx->rows, ctx->d_H,
-        ctx->d_V, ctx->d_P, ctx->d_status, layer, c.n_layers, c.n_q_heads, c.n_kv_heads,
-        1.0 / (double)c.tau1, 1.0 / (double)c.tau2);
+  if (finalize && !ctx->use_tc) {
+    finalize_layer<<<ctx->n_req, 128, 0, st>>>(ctx->d_colpart, ctx->d_req, ctx->d_H, ctx->d_V,
+                                                ctx->d_P, ctx->d_status, layer, c.n_layers,
+                                                c.n_q_heads, c.n_kv_heads, 1.0 / (double)c.tau1,
+                                                1.0 / (double)c.tau2);
     count_launch();
-    return cuda_status(cudaGetLastError());
   }
-  finalize_layer<<<ctx->n_req, 128, 0, st>>>(ctx->d_colpart, ctx->d_req, ctx->d_H, ctx->d_V,
-                                              ctx->d_P, ctx->d_status, layer, c.n_layers,
-                                              c.n_q_heads, c.n_kv_heads, 1.0 / (double)c.tau1,
-                                              1.0 / (double)c.tau2);
-  count_launch();
-  return cuda_status(cudaGetLastError());
-}
-
-int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, cudaStream_t st) {
-  const cake_config& c = ctx->cfg;
-  if (ctx->n_req == 0 || ctx->n_chunks == 0) return CAKE_OK;
-  const dim3 grid((unsigned)ctx->n_chunks, c.n_kv_heads);
-  pool_hist<<<grid, PH_THREADS, 0, st>>>(ctx->d_raw, ctx->d_fresh, ctx->d_req, ctx->d_chunks,
-                                         ctx->d_hist, ctx->d_arrivals, ctx->d_prefix, layer,
-                                         c.n_layers, c.n_kv_heads, ctx->total_tokens, c.pool_kernel,
-                                         c.pool_mode, do_pool ? 1 : 0);
+  FinalizeArgs F;
+  memset(&F, 0, sizeof(F));
+  F.Hq = c.n_q_heads;
+  if (finalize && ctx->use_tc) {
+    F.colpart = ctx->d_colpart;
+    F.pair_seg = ctx->d_tc_index + (ctx->n_req * c.n_kv_heads + 1);
+    F.hrow = ctx->d_hrow;
+    F.headsum = ctx->d_headsum;
+    F.fin_arrivals = ctx->d_arrivals + ctx->max_pairs;
+    F.dH = ctx->d_H; F.dV = ctx->d_V; F.dP = ctx->d_P;
+    F.status = ctx->d_status;
+    F.units = ctx->n_req * (c.n_q_heads / c.n_kv_heads);
+    F.use_hrow = ctx->hhead_from_rows ? 1 : 0;
+    F.rows = ctx->rows;
+    F.inv_tau1 = 1.0 / (double)c.tau1;
+    F.inv_tau2 = 1.0 / (double)c.tau2;
+  }
+  if (ctx->n_chunks + F.units == 0) return cuda_status(cudaGetLastError());
+  const dim3 grid((unsigned)(ctx->n_chunks + F.units), c.n_kv_heads);
+  const int r = c.pool_kernel / 2;
+#define CAKE_POOL_LAUNCH(RR)                                                                     \
+  pool_hist<RR><<<grid, PH_THREADS, 0, st>>>(ctx->d_raw, ctx->d_fresh, ctx->d_req, ctx->d_chunks, \
+                                             ctx->d_hist, ctx->d_arrivals, ctx->d_prefix,        \
+                                             ctx->n_chunks, layer, c.n_layers, c.n_kv_heads,     \
+                                             ctx->total_tokens, c.pool_kernel, c.pool_mode,      \
+                                             do_pool ? 1 : 0, F)
+  switch (r) {
+    case 0: CAKE_POOL_LAUNCH(0); break;
+    case 1: CAKE_POOL_LAUNCH(1); break;
+    case 2: CAKE_POOL_LAUNCH(2); break;
+    case 3: CAKE_POOL_LAUNCH(3); break;
+    default: CAKE_POOL_LAUNCH(-1); break;
+  }
+#undef CAKE_POOL_LAUNCH
   count_launch();
   return cuda_status(cudaGetLastError());
 }
