@@ -59,19 +59,27 @@ __global__ void budgets_with_window(const int32_t* __restrict__ b, int32_t* __re
 void free_ctx(cake_ctx* c) {
   if (!c) return;
   cudaFree(c->d_req); cudaFree(c->d_units); cudaFree(c->d_H); cudaFree(c->d_V); cudaFree(c->d_P);
-  cudaFree(c->d_budget[0]); cudaFree(c->d_budget[1]); cudaFree(c->d_status); cudaFree(c->d_raw);
+  cudaFree(c->d_budget[0]); cudaFree(c->d_budget[1]); cudaFree(c->d_status);
+  cudaFree(c->d_raw[0]); cudaFree(c->d_raw[1]);
   cudaFree(c->d_fresh); cudaFree(c->d_lists); cudaFree(c->d_prefix); cudaFree(c->d_lstate);
   cudaFree(c->d_hist); cudaFree(c->d_fill); cudaFree(c->d_arrivals); cudaFree(c->d_headsum); cudaFree(c->d_chunks);
   cudaFree(c->d_pos_packed); cudaFree(c->d_bitmap); cudaFree(c->d_lse2);
   if (c->h_chunks) cudaFreeHost(c->h_chunks);
-  cudaFree(c->d_rowpart); cudaFree(c->d_colpart);
+  cudaFree(c->d_rowpart); cudaFree(c->d_colpart[0]); cudaFree(c->d_colpart[1]);
   cudaFree(c->d_tc_ops); cudaFree(c->d_tc_index); cudaFree(c->d_tc_sync);
-  cudaFree(c->d_tc_rowpart); cudaFree(c->d_lse2_tc); cudaFree(c->d_hrow);
+  cudaFree(c->d_tc_rowpart); cudaFree(c->d_lse2_tc); cudaFree(c->d_hrow[0]); cudaFree(c->d_hrow[1]);
   if (c->h_tc_ops) cudaFreeHost(c->h_tc_ops);
   if (c->h_tc_index) cudaFreeHost(c->h_tc_index);
   if (c->h_req) cudaFreeHost(c->h_req);
   if (c->h_units) cudaFreeHost(c->h_units);
   if (c->upload_done) cudaEventDestroy(c->upload_done);
+  if (c->ev_main) cudaEventDestroy(c->ev_main);
+  if (c->ev_side) cudaEventDestroy(c->ev_side);
+  for (int i = 0; i < 2; ++i) {
+    if (c->ev_score[i]) cudaEventDestroy(c->ev_score[i]);
+    if (c->ev_tail[i]) cudaEventDestroy(c->ev_tail[i]);
+  }
+  if (c->side) cudaStreamDestroy(c->side);
   if (c->prof.spans) {
     for (int i = 0; i < c->prof.cap; ++i) {
       if (c->prof.spans[i].a) cudaEventDestroy(c->prof.spans[i].a);
@@ -81,6 +89,19 @@ void free_ctx(cake_ctx* c) {
   }
   free(c->h_cu);
   delete c;
+}
+
+// Orders the side stream after everything enqueued so far on the caller's stream.
+cudaError_t side_after(cake_ctx* c, cudaStream_t st) {
+  cudaError_t e = cudaEventRecord(c->ev_main, st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_main, 0);
+  return e;
+}
+// Orders the caller's stream after everything enqueued so far on the side stream.
+cudaError_t main_after_side(cake_ctx* c, cudaStream_t st) {
+  cudaError_t e = cudaEventRecord(c->ev_side, c->side);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_side, 0);
+  return e;
 }
 
 }  // namespace
@@ -120,6 +141,14 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   cudaError_t e = cudaGetDevice(&x->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&x->n_sm, cudaDevAttrMultiProcessorCount, x->device);
   if (e != cudaSuccess) { free_ctx(x); return CAKE_ERR_CUDA; }
+  {
+    // SMs left to the cascade kernels while a score kernel runs (CAKE_RESERVED_SMS, default 8)
+    int reserve = 8;
+    if (const char* env = getenv("CAKE_RESERVED_SMS")) reserve = atoi(env);
+    if (reserve < 0) reserve = 0;
+    if (reserve > x->n_sm / 2) reserve = x->n_sm / 2;
+    x->n_sm_score = x->n_sm - reserve;
+  }
 
   const int64_t T = c.max_total_tokens;
   const int64_t R = c.max_requests;
@@ -142,6 +171,13 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   ok = ok && cudaMallocHost((void**)&x->h_req, sizeof(ReqInfo) * R) == cudaSuccess;
   ok = ok && cudaMallocHost((void**)&x->h_units, sizeof(ScoreUnit) * x->max_units) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&x->upload_done, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&x->side, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&x->ev_main, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&x->ev_side, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; i < 2; ++i) {
+    ok = ok && cudaEventCreateWithFlags(&x->ev_score[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&x->ev_tail[i], cudaEventDisableTiming) == cudaSuccess;
+  }
   ok = ok && dev_alloc(&x->d_req, R) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_units, x->max_units) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_H, R * c.n_layers) == cudaSuccess;
@@ -150,7 +186,8 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   ok = ok && dev_alloc(&x->d_budget[0], R * c.n_layers) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_budget[1], R * c.n_layers) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_status, 1) == cudaSuccess;
-  ok = ok && dev_alloc(&x->d_raw, (size_t)c.n_kv_heads * T) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_raw[0], (size_t)c.n_kv_heads * T) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_raw[1], (size_t)c.n_kv_heads * T) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_fresh, (size_t)c.n_kv_heads * T) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_lists, (size_t)x->list_elems) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_prefix, (size_t)x->max_lists * (kBins + 1)) == cudaSuccess;
@@ -182,7 +219,8 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   }
   {
     const size_t a = (size_t)x->max_units * c.n_kv_heads, b = (size_t)x->max_tc_segs * kScoreWarps;
-    ok = ok && dev_alloc(&x->d_colpart, (a > b ? a : b) * G * 2) == cudaSuccess;
+    ok = ok && dev_alloc(&x->d_colpart[0], (a > b ? a : b) * G * 2) == cudaSuccess;
+    ok = ok && dev_alloc(&x->d_colpart[1], (a > b ? a : b) * G * 2) == cudaSuccess;
   }
   if (x->use_tc) {
     const size_t n_index = 2 * (size_t)(max_pairs + 1) + 2 * (size_t)(x->n_sm + 1);
@@ -193,7 +231,8 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
     ok = ok && dev_alloc(&x->d_tc_sync, 2 * (size_t)max_pairs) == cudaSuccess;
     ok = ok && dev_alloc(&x->d_tc_rowpart, (size_t)x->max_tc_segs * kScoreGroups * 128) == cudaSuccess;
     ok = ok && dev_alloc(&x->d_lse2_tc, (size_t)max_pairs * 128) == cudaSuccess;
-    ok = ok && dev_alloc(&x->d_hrow, (size_t)max_pairs * 128) == cudaSuccess;
+    ok = ok && dev_alloc(&x->d_hrow[0], (size_t)max_pairs * 128) == cudaSuccess;
+    ok = ok && dev_alloc(&x->d_hrow[1], (size_t)max_pairs * 128) == cudaSuccess;
   }
   ok = ok && cudaMemset(x->d_status, 0, sizeof(int32_t)) == cudaSuccess;
   ok = ok && cudaMemset(x->d_budget[0], 0, sizeof(int32_t) * R * c.n_layers) == cudaSuccess;
@@ -225,6 +264,8 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
       if (cu[r + 1] - cu[r] < c.window) return CAKE_ERR_ARG;
     if (cu[n_req] > c.max_total_tokens) return CAKE_ERR_CAPACITY;
   }
+  // the previous batch's cascade must be done before its state is reset or overwritten
+  CAKE_CUDA_TRY(main_after_side(ctx, st));
   const int64_t T = n_req > 0 ? cu[n_req] : 0;
   const bool same = ctx->n_req == n_req && n_req > 0 &&
                     memcmp(ctx->h_cu, cu, sizeof(int64_t) * (n_req + 1)) == 0;
@@ -296,6 +337,8 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
   ctx->alloc_of_buf[0] = ctx->alloc_of_buf[1] = -1;
   ctx->last_alloc = -1;
   CAKE_CUDA_TRY(cudaMemsetAsync(ctx->d_status, 0, sizeof(int32_t), st));
+  ctx->tail_recorded[0] = ctx->tail_recorded[1] = false;
+  CAKE_CUDA_TRY(side_after(ctx, st));
   return CAKE_OK;
 }
 
@@ -306,12 +349,18 @@ int32_t cake_score_layer(cake_ctx* ctx, int32_t layer, const void* q_win, const 
   if (ctx->n_req > 0 && (!q_win || !k)) return CAKE_ERR_ARG;
   if (layer != ctx->n_ind || ctx->n_evicted != layer) return CAKE_ERR_STATE;
   cudaStream_t st = (cudaStream_t)stream;
-  int32_t rc = ctx->use_tc ? launch_score_tc(ctx, q_win, k, lse, st)
-                           : launch_score_simt(ctx, q_win, k, lse, st);
+  const int par = layer & 1;
+  // the buffers of this parity were last read by the cascade of layer - 2
+  if (ctx->tail_recorded[par]) CAKE_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev_tail[par], 0));
+  int32_t rc = ctx->use_tc ? launch_score_tc(ctx, layer, q_win, k, lse, st)
+                           : launch_score_simt(ctx, layer, q_win, k, lse, st);
   if (rc != CAKE_OK) return rc;
-  const int sp = prof_begin(ctx, CAKE_PROF_FINALIZE, st);
-  rc = launch_pool(ctx, layer, true, true, st);
-  prof_end(ctx, sp, st);
+  // everything after the score kernel runs on the side stream, beside the next layer's scoring
+  CAKE_CUDA_TRY(cudaEventRecord(ctx->ev_score[par], st));
+  CAKE_CUDA_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_score[par], 0));
+  const int sp = prof_begin(ctx, CAKE_PROF_FINALIZE, ctx->side);
+  rc = launch_pool(ctx, layer, true, true, ctx->side);
+  prof_end(ctx, sp, ctx->side);
   if (rc != CAKE_OK) return rc;
   ctx->n_ind = layer + 1;
   if (ctx->n_pref < layer + 1) ctx->n_pref = layer + 1;
@@ -322,9 +371,10 @@ int32_t cake_allocate(cake_ctx* ctx, int32_t stage, void* stream) {
   if (!ctx || ctx->n_req < 0) return ctx ? CAKE_ERR_STATE : CAKE_ERR_ARG;
   if (stage < 0 || stage >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
   if (stage >= ctx->n_pref) return CAKE_ERR_STATE;
-  const int sp = prof_begin(ctx, CAKE_PROF_ALLOCATE, (cudaStream_t)stream);
-  int32_t rc = launch_allocate(ctx, stage, (cudaStream_t)stream);
-  prof_end(ctx, sp, (cudaStream_t)stream);
+  (void)stream;                      // ordered by the side stream
+  const int sp = prof_begin(ctx, CAKE_PROF_ALLOCATE, ctx->side);
+  int32_t rc = launch_allocate(ctx, stage, ctx->side);
+  prof_end(ctx, sp, ctx->side);
   if (rc != CAKE_OK) return rc;
   ctx->alloc_of_buf[stage & 1] = stage;
   ctx->last_alloc = stage;
@@ -337,10 +387,13 @@ int32_t cake_evict(cake_ctx* ctx, int32_t stage, void* stream) {
   if (stage != ctx->n_evicted || ctx->n_ind != stage + 1) return CAKE_ERR_STATE;
   if (ctx->alloc_of_buf[stage & 1] != stage) return CAKE_ERR_STATE;
   if (stage > 0 && ctx->alloc_of_buf[(stage + 1) & 1] != stage - 1) return CAKE_ERR_STATE;
-  const int sp = prof_begin(ctx, CAKE_PROF_EVICT, (cudaStream_t)stream);
-  int32_t rc = launch_evict(ctx, stage, (cudaStream_t)stream);
-  prof_end(ctx, sp, (cudaStream_t)stream);
+  (void)stream;
+  const int sp = prof_begin(ctx, CAKE_PROF_EVICT, ctx->side);
+  int32_t rc = launch_evict(ctx, stage, ctx->side);
+  prof_end(ctx, sp, ctx->side);
   if (rc != CAKE_OK) return rc;
+  CAKE_CUDA_TRY(cudaEventRecord(ctx->ev_tail[stage & 1], ctx->side));
+  ctx->tail_recorded[stage & 1] = true;
   ctx->n_evicted = stage + 1;
   return CAKE_OK;
 }
@@ -363,6 +416,7 @@ int32_t cake_compact(cake_ctx* ctx, int32_t layer_lo, int32_t layer_hi, const vo
       ptrs.v[l] = v_layers[l];
     }
   }
+  CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
   const int sp = prof_begin(ctx, CAKE_PROF_COMPACT, (cudaStream_t)stream);
   const int32_t rc = launch_compact(ctx, layer_lo, layer_hi, ptrs, k_out, v_out, row_offsets_out,
                                     positions_out, (cudaStream_t)stream);
@@ -380,6 +434,7 @@ int32_t cake_get_indicators(cake_ctx* ctx, int32_t layer, float* out, void* stre
   if (!ctx || !out) return CAKE_ERR_ARG;
   if (ctx->n_req < 0 || layer != ctx->n_ind - 1) return CAKE_ERR_STATE;
   if (ctx->total_tokens == 0) return CAKE_OK;
+  CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
   CAKE_CUDA_TRY(cudaMemcpyAsync(out, ctx->d_fresh,
                                 sizeof(float) * ctx->cfg.n_kv_heads * ctx->total_tokens,
                                 cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
@@ -392,6 +447,7 @@ int32_t cake_get_preferences(cake_ctx* ctx, double* H, double* V, double* P, voi
   const size_t bytes = sizeof(double) * ctx->n_req * ctx->cfg.n_layers;
   cudaStream_t st = (cudaStream_t)stream;
   if (bytes == 0) return CAKE_OK;
+  CAKE_CUDA_TRY(main_after_side(ctx, st));
   if (H) CAKE_CUDA_TRY(cudaMemcpyAsync(H, ctx->d_H, bytes, cudaMemcpyDeviceToDevice, st));
   if (V) CAKE_CUDA_TRY(cudaMemcpyAsync(V, ctx->d_V, bytes, cudaMemcpyDeviceToDevice, st));
   if (P) CAKE_CUDA_TRY(cudaMemcpyAsync(P, ctx->d_P, bytes, cudaMemcpyDeviceToDevice, st));
@@ -403,12 +459,15 @@ int32_t cake_set_indicators(cake_ctx* ctx, int32_t layer, const float* in, void*
   if (ctx->n_req < 0) return CAKE_ERR_STATE;
   if (layer < 0 || layer >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
   if (layer != ctx->n_ind || ctx->n_evicted != layer) return CAKE_ERR_STATE;
+  // the previous stage may still read the pooled buffer on the side stream
+  CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
   if (ctx->total_tokens > 0)
     CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_fresh, in,
                                   sizeof(float) * ctx->cfg.n_kv_heads * ctx->total_tokens,
                                   cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  CAKE_CUDA_TRY(side_after(ctx, (cudaStream_t)stream));
   // bucket histogram of the supplied values (they are taken as already pooled)
-  const int32_t rc = launch_pool(ctx, layer, false, false, (cudaStream_t)stream);
+  const int32_t rc = launch_pool(ctx, layer, false, false, ctx->side);
   if (rc != CAKE_OK) return rc;
   ctx->n_ind = layer + 1;
   return CAKE_OK;
@@ -418,10 +477,13 @@ int32_t cake_set_preferences(cake_ctx* ctx, int32_t n_set, const double* P, void
   if (!ctx || !P) return CAKE_ERR_ARG;
   if (ctx->n_req < 0) return CAKE_ERR_STATE;
   if (n_set < 1 || n_set > ctx->cfg.n_layers) return CAKE_ERR_ARG;
-  if (ctx->n_req > 0)
+  if (ctx->n_req > 0) {
+    CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
     CAKE_CUDA_TRY(cudaMemcpy2DAsync(ctx->d_P, sizeof(double) * ctx->cfg.n_layers, P,
                                     sizeof(double) * n_set, sizeof(double) * n_set, ctx->n_req,
                                     cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    CAKE_CUDA_TRY(side_after(ctx, (cudaStream_t)stream));
+  }
   if (ctx->n_pref < n_set) ctx->n_pref = n_set;
   return CAKE_OK;
 }
@@ -431,6 +493,7 @@ int32_t cake_get_budgets(cake_ctx* ctx, int32_t* out, void* stream) {
   if (ctx->n_req < 0 || ctx->last_alloc < 0) return CAKE_ERR_STATE;
   if (ctx->n_req == 0) return CAKE_OK;
   const int total = ctx->n_req * ctx->cfg.n_layers;
+  CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
   budgets_with_window<<<(total + 127) / 128, 128, 0, (cudaStream_t)stream>>>(
       ctx->d_budget[ctx->last_alloc & 1], out, ctx->n_req, ctx->cfg.n_layers, ctx->last_alloc + 1,
       ctx->cfg.window);
@@ -444,6 +507,7 @@ int32_t cake_get_positions(cake_ctx* ctx, int32_t req, int32_t layer, int32_t* o
   if (ctx->n_req < 0) return CAKE_ERR_STATE;
   if (req < 0 || req >= ctx->n_req || layer < 0 || layer >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
   if (layer >= ctx->n_evicted || ctx->last_alloc != ctx->n_evicted - 1) return CAKE_ERR_STATE;
+  CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
   return launch_get_positions(ctx, req, layer, out, capacity, (cudaStream_t)stream);
 }
 
@@ -451,6 +515,7 @@ int32_t cake_status(cake_ctx* ctx, int32_t* device_status_out, void* stream) {
   if (!ctx) return CAKE_ERR_ARG;
   int32_t s = 0;
   cudaStream_t st = (cudaStream_t)stream;
+  CAKE_CUDA_TRY(main_after_side(ctx, st));
   CAKE_CUDA_TRY(cudaMemcpyAsync(&s, ctx->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
   CAKE_CUDA_TRY(cudaStreamSynchronize(st));
   if (device_status_out) *device_status_out = s;
@@ -471,6 +536,7 @@ int32_t cake_profile_enable(cake_ctx* ctx, int32_t on) {
 
 int32_t cake_profile_read(cake_ctx* ctx, double* ms_out, int64_t* spans_out, void* stream) {
   if (!ctx || !ms_out || !spans_out) return CAKE_ERR_ARG;
+  CAKE_CUDA_TRY(cudaStreamSynchronize(ctx->side));
   CAKE_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
   for (int k = 0; k < CAKE_PROF_KINDS; ++k) { ms_out[k] = 0.0; spans_out[k] = 0; }
   Profiler& p = ctx->prof;

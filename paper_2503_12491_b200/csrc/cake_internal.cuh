@@ -85,6 +85,15 @@ struct cake_ctx {
   cake::Profiler prof;
   int device;
   int n_sm;
+  int n_sm_score;          // SMs the persistent score kernel occupies; the rest stay free for the
+                           // cascade kernels of the previous layer, which run beside it
+  // The cascade of layer l (pooling, preference, budgets, eviction) runs on an internal side
+  // stream while the caller's stream already scores layer l+1; events order the two.
+  cudaStream_t side;
+  cudaEvent_t ev_main, ev_side;     // scratch events: caller's stream -> side, side -> caller's
+  cudaEvent_t ev_score[2];          // score kernel of a layer of that parity has finished
+  cudaEvent_t ev_tail[2];           // eviction stage of that parity has finished
+  bool tail_recorded[2];
   int32_t rows;            // R = G * S_w
   int64_t sel_budget;      // B' = B_total - L * S_w
   // ---- batch state (host) ----
@@ -112,7 +121,7 @@ struct cake_ctx {
   double* d_P;
   int32_t* d_budget[2];    // [max_requests][L] selectable budgets, double-buffered by stage parity
   int32_t* d_status;       // sticky device status word
-  float* d_raw;            // [H_kv][max_total_tokens] un-pooled indicator
+  float* d_raw[2];         // [H_kv][max_total_tokens] un-pooled indicator, by layer parity
   float* d_fresh;          // [H_kv][max_total_tokens] pooled indicator of the newest layer
   uint2* d_lists;          // per (req, layer, head): n entries (ordered indicator key, position)
   int64_t list_elems;
@@ -132,7 +141,7 @@ struct cake_ctx {
   int64_t bitmap_words;
   float* d_lse2;           // [max_requests][H_q][S_w] base-2 log-sum-exp of window rows
   float2* d_rowpart;       // [max_units][H_kv][R] (max, sum) partials of phase A
-  float* d_colpart;        // [max_units][H_kv][G][2] partial (sum p*log2 p, sum var) of phase B
+  float* d_colpart[2];     // partial (sum p*log2 p, sum var) of the column pass, by layer parity
   // ---- tensor-core score path ----
   bool use_tc;
   bool hhead_from_rows;    // entropy came from pass A (d_hrow) rather than from pass B partials
@@ -150,7 +159,7 @@ struct cake_ctx {
   uint32_t* d_tc_sync;            // [max_pairs] delivered partial rows, then [max_pairs] merged rows
   float4* d_tc_rowpart;           // [max_tc_segs][kScoreGroups][128]
   float* d_lse2_tc;               // [max_requests][H_kv][128], rows in tile order i*G + h
-  float* d_hrow;                  // [max_pairs][128] sum_j p log2 p per window row from pass A
+  float* d_hrow[2];               // [max_pairs][128] sum_j p log2 p per window row, by layer parity
 };
 
 namespace cake {
@@ -158,14 +167,14 @@ namespace cake {
 void count_launch(int64_t n = 1);
 
 // score_simt.cu
-int32_t launch_score_simt(cake_ctx* ctx, const void* q_win, const void* k, const float* lse,
-                          cudaStream_t st);
+int32_t launch_score_simt(cake_ctx* ctx, int32_t layer, const void* q_win, const void* k,
+                          const float* lse, cudaStream_t st);
 // score_tc.cu
 bool tc_path_supported(const cake_config& c);
 int64_t tc_max_segments(const cake_config& c, int n_sm);
 int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req);
-int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const float* lse,
-                        cudaStream_t st);
+int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const void* k,
+                        const float* lse, cudaStream_t st);
 // cascade.cu
 int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, bool finalize, cudaStream_t st);
 int32_t launch_allocate(cake_ctx* ctx, int32_t stage, cudaStream_t st);

@@ -711,7 +711,7 @@ int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, bool finalize, c
   const cake_config& c = ctx->cfg;
   if (ctx->n_req == 0) return CAKE_OK;
   if (finalize && !ctx->use_tc) {
-    finalize_layer<<<ctx->n_req, 128, 0, st>>>(ctx->d_colpart, ctx->d_req, ctx->d_H, ctx->d_V,
+    finalize_layer<<<ctx->n_req, 128, 0, st>>>(ctx->d_colpart[layer & 1], ctx->d_req, ctx->d_H, ctx->d_V,
                                                 ctx->d_P, ctx->d_status, layer, c.n_layers,
                                                 c.n_q_heads, c.n_kv_heads, 1.0 / (double)c.tau1,
                                                 1.0 / (double)c.tau2);
@@ -721,9 +721,9 @@ int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, bool finalize, c
   memset(&F, 0, sizeof(F));
   F.Hq = c.n_q_heads;
   if (finalize && ctx->use_tc) {
-    F.colpart = ctx->d_colpart;
+    F.colpart = ctx->d_colpart[layer & 1];
     F.pair_seg = ctx->d_tc_index + (ctx->n_req * c.n_kv_heads + 1);
-    F.hrow = ctx->d_hrow;
+    F.hrow = ctx->d_hrow[layer & 1];
     F.headsum = ctx->d_headsum;
     F.fin_arrivals = ctx->d_arrivals + ctx->max_pairs;
     F.dH = ctx->d_H; F.dV = ctx->d_V; F.dP = ctx->d_P;
@@ -738,7 +738,7 @@ int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, bool finalize, c
   const dim3 grid((unsigned)(ctx->n_chunks + F.units), c.n_kv_heads);
   const int r = c.pool_kernel / 2;
 #define CAKE_POOL_LAUNCH(RR)                                                                     \
-  pool_hist<RR><<<grid, PH_THREADS, 0, st>>>(ctx->d_raw, ctx->d_fresh, ctx->d_req, ctx->d_chunks, \
+  pool_hist<RR><<<grid, PH_THREADS, 0, st>>>(ctx->d_raw[layer & 1], ctx->d_fresh, ctx->d_req, ctx->d_chunks, \
                                              ctx->d_hist, ctx->d_arrivals, ctx->d_prefix,        \
                                              ctx->n_chunks, layer, c.n_layers, c.n_kv_heads,     \
                                              ctx->total_tokens, c.pool_kernel, c.pool_mode,      \

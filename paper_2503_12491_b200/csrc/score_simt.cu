@@ -319,7 +319,8 @@ score_colstats_simt(const T* __restrict__ q_win, const T* __restrict__ k,
 }
 
 template <typename T>
-int32_t run(cake_ctx* ctx, const void* q_win, const void* k, const float* lse, cudaStream_t st) {
+int32_t run(cake_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* lse,
+            cudaStream_t st) {
   const cake_config& c = ctx->cfg;
   const int rows = ctx->rows;
   const size_t smem = smem_bytes(rows, c.head_dim);
@@ -350,8 +351,8 @@ int32_t run(cake_ctx* ctx, const void* q_win, const void* k, const float* lse, c
   prof_end(ctx, sp, st);
   sp = prof_begin(ctx, CAKE_PROF_SCORE, st);
   score_colstats_simt<T><<<grid, NT, smem, st>>>(
-      (const T*)q_win, (const T*)k, ctx->d_req, ctx->d_units, ctx->d_lse2, ctx->d_raw,
-      ctx->d_colpart, c.n_q_heads, c.n_kv_heads, c.window, c.head_dim, ctx->total_tokens, scale2,
+      (const T*)q_win, (const T*)k, ctx->d_req, ctx->d_units, ctx->d_lse2, ctx->d_raw[layer & 1],
+      ctx->d_colpart[layer & 1], c.n_q_heads, c.n_kv_heads, c.window, c.head_dim, ctx->total_tokens, scale2,
       c.gamma, c.var_ddof);
   count_launch();
   prof_end(ctx, sp, st);
@@ -360,11 +361,11 @@ int32_t run(cake_ctx* ctx, const void* q_win, const void* k, const float* lse, c
 
 }  // namespace
 
-int32_t launch_score_simt(cake_ctx* ctx, const void* q_win, const void* k, const float* lse,
-                          cudaStream_t st) {
+int32_t launch_score_simt(cake_ctx* ctx, int32_t layer, const void* q_win, const void* k,
+                          const float* lse, cudaStream_t st) {
   if (ctx->n_units == 0) return CAKE_OK;
-  if (ctx->cfg.dtype == CAKE_DTYPE_FP32) return run<float>(ctx, q_win, k, lse, st);
-  return run<__nv_bfloat16>(ctx, q_win, k, lse, st);
+  if (ctx->cfg.dtype == CAKE_DTYPE_FP32) return run<float>(ctx, layer, q_win, k, lse, st);
+  return run<__nv_bfloat16>(ctx, layer, q_win, k, lse, st);
 }
 
 }  // namespace cake

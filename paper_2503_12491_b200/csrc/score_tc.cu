@@ -820,7 +820,7 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
   const int64_t T = n_req > 0 ? ctx->h_req[n_req - 1].cu + ctx->h_req[n_req - 1].N : 0;
   int64_t tilesA_total = 0;
   for (int r = 0; r < n_req; ++r) tilesA_total += (int64_t)Hkv * ((ctx->h_req[r].N + TILE - 1) / TILE);
-  const int n_cta = (int)(tilesA_total < ctx->n_sm ? tilesA_total : ctx->n_sm);
+  const int n_cta = (int)(tilesA_total < ctx->n_sm_score ? tilesA_total : ctx->n_sm_score);
   ctx->n_tc_ctas = n_cta;
   ctx->n_tc_ops_full = ctx->n_tc_ops_b = 0;
   ctx->n_tc_asegs = ctx->n_tc_bsegs = 0;
@@ -898,8 +898,8 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
   return CAKE_OK;
 }
 
-int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const float* lse,
-                        cudaStream_t st) {
+int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const void* k,
+                        const float* lse, cudaStream_t st) {
   const cake_config& c = ctx->cfg;
   if (ctx->n_tc_ctas == 0) return CAKE_OK;
   if ((int64_t)c.n_kv_heads * ctx->total_tokens >= ((int64_t)1 << 31)) return CAKE_ERR_ARG;
@@ -938,9 +938,9 @@ int32_t launch_score_tc(cake_ctx* ctx, const void* q_win, const void* k, const f
   P.pair_cnt = ctx->d_tc_sync;
   P.lse2 = ctx->d_lse2_tc;
   P.rowpart = ctx->d_tc_rowpart;
-  P.raw = ctx->d_raw;
-  P.colpart = ctx->d_colpart;
-  P.hrow = ctx->d_hrow;
+  P.raw = ctx->d_raw[layer & 1];
+  P.colpart = ctx->d_colpart[layer & 1];
+  P.hrow = ctx->d_hrow[layer & 1];
   P.n_pairs = n_pairs;
   P.status = ctx->d_status;
   P.T = ctx->total_tokens;
