@@ -62,9 +62,8 @@ void free_ctx(cake_ctx* c) {
   cudaFree(c->d_budget[0]); cudaFree(c->d_budget[1]); cudaFree(c->d_status);
   cudaFree(c->d_raw[0]); cudaFree(c->d_raw[1]);
   cudaFree(c->d_fresh); cudaFree(c->d_lists); cudaFree(c->d_prefix); cudaFree(c->d_lstate);
-  cudaFree(c->d_hist); cudaFree(c->d_fill); cudaFree(c->d_arrivals); cudaFree(c->d_headsum); cudaFree(c->d_chunks);
+  cudaFree(c->d_hist); cudaFree(c->d_fill); cudaFree(c->d_arrivals); cudaFree(c->d_headsum);
   cudaFree(c->d_pos_packed); cudaFree(c->d_bitmap); cudaFree(c->d_lse2);
-  if (c->h_chunks) cudaFreeHost(c->h_chunks);
   cudaFree(c->d_rowpart); cudaFree(c->d_colpart[0]); cudaFree(c->d_colpart[1]);
   cudaFree(c->d_tc_ops); cudaFree(c->d_tc_index); cudaFree(c->d_tc_sync);
   cudaFree(c->d_tc_rowpart); cudaFree(c->d_lse2_tc); cudaFree(c->d_hrow[0]); cudaFree(c->d_hrow[1]);
@@ -142,8 +141,8 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&x->n_sm, cudaDevAttrMultiProcessorCount, x->device);
   if (e != cudaSuccess) { free_ctx(x); return CAKE_ERR_CUDA; }
   {
-    // SMs left to the cascade kernels while a score kernel runs (CAKE_RESERVED_SMS, default 8)
-    int reserve = 8;
+    // SMs left to the cascade kernels while a score kernel runs (CAKE_RESERVED_SMS, default 16)
+    int reserve = 16;
     if (const char* env = getenv("CAKE_RESERVED_SMS")) reserve = atoi(env);
     if (reserve < 0) reserve = 0;
     if (reserve > x->n_sm / 2) reserve = x->n_sm / 2;
@@ -156,7 +155,6 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   x->max_units = (int32_t)(T / kSimtTileKeys + R + 1);
   x->list_elems = T * c.n_layers * c.n_kv_heads;
   x->max_lists = R * c.n_layers * c.n_kv_heads;
-  x->max_chunks = (int32_t)(T / kChunkKeys + R + 1);
   {
     // packed rows: H_kv * sum_r min(B_total, L * N_r) <= H_kv * min(R * B_total, L * T)
     const int64_t a = R * c.total_budget, b = (int64_t)c.n_layers * T;
@@ -196,10 +194,8 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   ok = ok && dev_alloc(&x->d_fill, (size_t)R * c.n_kv_heads * kBins) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_arrivals, (size_t)R * c.n_kv_heads + R) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_headsum, (size_t)R * c.n_q_heads * 2) == cudaSuccess;
-  ok = ok && dev_alloc(&x->d_chunks, (size_t)x->max_chunks) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_pos_packed, (size_t)x->pos_packed_cap) == cudaSuccess;
   if (x->bitmap_words > 0) ok = ok && dev_alloc(&x->d_bitmap, (size_t)x->bitmap_words) == cudaSuccess;
-  ok = ok && cudaMallocHost((void**)&x->h_chunks, sizeof(ScoreUnit) * x->max_chunks) == cudaSuccess;
   ok = ok && cudaMemset(x->d_hist, 0, sizeof(uint32_t) * R * c.n_kv_heads * kBins) == cudaSuccess;
   ok = ok && cudaMemset(x->d_fill, 0, sizeof(uint32_t) * R * c.n_kv_heads * kBins) == cudaSuccess;
   ok = ok && cudaMemset(x->d_arrivals, 0, sizeof(uint32_t) * (R * c.n_kv_heads + R)) == cudaSuccess;
@@ -275,7 +271,12 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
       ctx->upload_pending = false;
     }
     const int32_t unit_keys = choose_unit_keys(T, c.n_kv_heads, ctx->n_sm);
-    int32_t nu = 0, nch = 0;
+    int32_t nu = 0, max_split = 0;
+    // the pooling / scatter kernels run on the SMs the score kernel leaves free: about two CTAs
+    // per such SM over all (request, head) pairs
+    const int reserve = ctx->n_sm - ctx->n_sm_score;
+    int want_split = (2 * (reserve > 0 ? reserve : 8)) / (n_req * c.n_kv_heads);
+    if (want_split < 1) want_split = 1;
     int64_t list_off = 0, bound = 0;
     for (int r = 0; r < n_req; ++r) {
       ReqInfo& q = ctx->h_req[r];
@@ -285,11 +286,12 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
       q.keep_all = q.N <= c.total_budget / c.n_layers ? 1 : 0;
       q.list_off = list_off;
       list_off += (int64_t)q.n * c.n_layers * c.n_kv_heads;
-      q.nchunks = 0;
-      for (int32_t k0 = 0; k0 < q.N; k0 += kChunkKeys) {
-        ScoreUnit& u = ctx->h_chunks[nch++];
-        u.req = r; u.key0 = k0; u.nkeys = q.N - k0 < kChunkKeys ? q.N - k0 : kChunkKeys; u.pad = 0;
-        ++q.nchunks;
+      {
+        const int chunks = (q.N + kChunkKeys - 1) / kChunkKeys;
+        int ns = chunks < want_split ? chunks : want_split;
+        q.span = ((chunks + ns - 1) / ns) * kChunkKeys;
+        q.nsplit = (q.N + q.span - 1) / q.span;
+        if (q.nsplit > max_split) max_split = q.nsplit;
       }
       q.unit0 = nu;
       for (int32_t k0 = 0; k0 < q.N; k0 += unit_keys) {
@@ -300,8 +302,8 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
       const int64_t full = (int64_t)c.n_layers * q.N;
       bound += (int64_t)c.n_kv_heads * (c.total_budget < full ? c.total_budget : full);
     }
-    if (list_off > ctx->list_elems || nu > ctx->max_units || nch > ctx->max_chunks) return CAKE_ERR_CAPACITY;
-    ctx->n_chunks = nch;
+    if (list_off > ctx->list_elems || nu > ctx->max_units) return CAKE_ERR_CAPACITY;
+    ctx->n_split = max_split;
     if (ctx->use_tc) {
       const int32_t prc = tc_build_plan(ctx, n_req);
       if (prc != CAKE_OK) return prc;
@@ -312,8 +314,6 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
     CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_req, ctx->h_req, sizeof(ReqInfo) * n_req,
                                   cudaMemcpyHostToDevice, st));
     CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_units, ctx->h_units, sizeof(ScoreUnit) * nu,
-                                  cudaMemcpyHostToDevice, st));
-    CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_chunks, ctx->h_chunks, sizeof(ScoreUnit) * nch,
                                   cudaMemcpyHostToDevice, st));
     if (ctx->use_tc && ctx->n_tc_ctas > 0) {
       const size_t n_index = 2 * (size_t)(n_req * c.n_kv_heads + 1) + 2 * (size_t)(ctx->n_sm + 1);
@@ -326,7 +326,7 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
     CAKE_CUDA_TRY(cudaEventRecord(ctx->upload_done, st));
     ctx->upload_pending = true;
   }
-  if (n_req == 0) { ctx->n_units = 0; ctx->n_chunks = 0; ctx->packed_rows_bound = 0; ctx->n_tc_ctas = 0; }
+  if (n_req == 0) { ctx->n_units = 0; ctx->n_split = 0; ctx->packed_rows_bound = 0; ctx->n_tc_ctas = 0; }
   if (ctx->use_tc) {
     ctx->tc_epoch = 0;
     CAKE_CUDA_TRY(cudaMemsetAsync(ctx->d_tc_sync, 0, sizeof(uint32_t) * 2 * ctx->max_pairs, st));

@@ -14,7 +14,7 @@ constexpr int kSimtTileKeys = 64;    // keys per tile of the SIMT score kernels
 constexpr int kSimtThreads = 256;
 constexpr int kBinBits = 12;         // survivor lists are sorted by the top bits of the indicator
 constexpr int kBins = 1 << kBinBits;
-constexpr int kChunkKeys = 4096;     // tokens per CTA of the pooling / scatter kernels
+constexpr int kChunkKeys = 4096;     // granularity of the token ranges of the pooling / scatter CTAs
 constexpr int kBitmapSmemWords = 48 * 1024;   // positions of up to 1.5 M tokens are ordered in shared memory
 constexpr int kScoreGroups = 3;      // statistics warp groups per CTA of the tensor-core score kernel
 constexpr int kScoreWarps = 4 * kScoreGroups;   // statistics warps: one column-pass partial each
@@ -25,7 +25,8 @@ struct ReqInfo {
   int32_t N;         // prompt length
   int32_t n;         // N - S_w non-window tokens
   int32_t keep_all;  // 1: N <= floor(B_total/L), nothing is evicted
-  int32_t nchunks;   // chunks of kChunkKeys tokens covering the prompt
+  int32_t nsplit;    // CTAs of the pooling / scatter kernels that share the prompt's tokens
+  int32_t span;      // tokens per such CTA (a multiple of kChunkKeys)
   int64_t list_off;  // first entry of this request's lists; list (layer, head) holds n entries
   int32_t unit0;     // first score unit of the request
   int32_t nunits;    // number of score units of the request
@@ -132,9 +133,7 @@ struct cake_ctx {
   uint32_t* d_fill;        // [max_pairs][kBins] scatter cursors (zero at rest)
   uint32_t* d_arrivals;    // [max_pairs] chunk counters, then [max_requests] head counters (zero at rest)
   double* d_headsum;       // [max_requests][H_q][2] per-head entropy / variance sums of the layer
-  cake::ScoreUnit* h_chunks;   // pinned
-  cake::ScoreUnit* d_chunks;
-  int32_t n_chunks, max_chunks;
+  int32_t n_split;         // largest nsplit of the batch
   int32_t* d_pos_packed;   // [packed rows bound] positions in packed row order
   int64_t pos_packed_cap;
   uint32_t* d_bitmap;      // global bitmaps for requests too long for shared memory (or null)

@@ -102,8 +102,8 @@ __device__ inline int block_excl_scan(int v, int* warp_tot, int* total) {
   return r;
 }
 
-constexpr int PH_THREADS = 256;
-constexpr int PH_PER = kChunkKeys / PH_THREADS;      // consecutive tokens per thread
+constexpr int PH_THREADS = 1024;
+constexpr int PH_PER = 4;                            // consecutive tokens per thread and pass
 
 struct FinalizeArgs {        // preference of the layer from the tensor-core kernel's partials
   const float* colpart;      // [pass-B segment][statistics warp][G][2]
@@ -113,7 +113,7 @@ struct FinalizeArgs {        // preference of the layer from the tensor-core ker
   uint32_t* fin_arrivals;    // [req], zero at rest
   double* dH; double* dV; double* dP;
   int32_t* status;
-  int units;                 // extra CTAs per KV head: n_req * G (0 = none)
+  int units;                 // extra CTAs per (KV head, request): G (0 = none)
   int use_hrow, rows, Hq;
   double inv_tau1, inv_tau2;
 };
@@ -170,92 +170,94 @@ __device__ void finalize_head(const FinalizeArgs& F, int req, int g, int hl, int
   }
 }
 
-// One CTA per (chunk of kChunkKeys tokens, KV head); a thread owns PH_PER consecutive tokens.
-// fresh[g][t] = pool(raw[g][.]) over the request's non-window tokens, +inf on the window
-// (Section 4.3); with do_pool = 0 the pooled values are already in `fresh`.  The bucket
-// histogram of the (request, head) is accumulated in `hist`; the CTA that adds the last chunk
-// turns it into the list's bucket offsets.  R = pool_kernel / 2 when that is at most 3, else
-// -1 (any kernel size, one global read per tap).  CTAs past the chunks finalise the layer's
-// preference (tensor-core path).
+// One CTA per (split of a request's tokens, KV head, request); a thread owns PH_PER consecutive
+// tokens per pass.  fresh[g][t] = pool(raw[g][.]) over the request's non-window tokens, +inf on
+// the window (Section 4.3); with do_pool = 0 the pooled values are already in `fresh`.  The
+// bucket histogram of the (request, head) is accumulated in `hist`; the CTA that adds the last
+// split turns it into the list's bucket offsets.  R = pool_kernel / 2 when that is at most 3,
+// else -1 (any kernel size, one global read per tap).  CTAs with blockIdx.x >= n_split finalise
+// the layer's preference (tensor-core path).  The grid is small on purpose: it runs on the few
+// SMs the score kernel of the next layer leaves free.
 template <int R>
 __global__ void __launch_bounds__(PH_THREADS)
 pool_hist(const float* __restrict__ raw, float* __restrict__ fresh, const ReqInfo* __restrict__ reqs,
-          const ScoreUnit* __restrict__ chunks, uint32_t* __restrict__ hist,
-          uint32_t* __restrict__ arrivals, int32_t* __restrict__ prefix, int n_chunks, int layer,
-          int L, int Hkv, int64_t T, int kp, int mode, int do_pool, const FinalizeArgs F) {
-  if ((int)blockIdx.x >= n_chunks) {
-    const int ex = (int)blockIdx.x - n_chunks, G = F.Hq / Hkv;
-    finalize_head(F, ex / G, blockIdx.y, ex % G, layer, L, Hkv);
+          uint32_t* __restrict__ hist, uint32_t* __restrict__ arrivals, int32_t* __restrict__ prefix,
+          int n_split, int layer, int L, int Hkv, int64_t T, int kp, int mode, int do_pool,
+          const FinalizeArgs F) {
+  const int g = blockIdx.y, req = blockIdx.z;
+  if ((int)blockIdx.x >= n_split) {
+    finalize_head(F, req, g, (int)blockIdx.x - n_split, layer, L, Hkv);
     return;
   }
   __shared__ uint32_t sh[kBins];
   __shared__ int warp_tot[32];
   __shared__ int s_total, s_last;
-  const ScoreUnit ch = chunks[blockIdx.x];
-  const int g = blockIdx.y;
-  const ReqInfo rq = reqs[ch.req];
-  const int pair = ch.req * Hkv + g;
+  const ReqInfo rq = reqs[req];
+  if ((int)blockIdx.x >= rq.nsplit) return;
+  const int pair = req * Hkv + g;
   for (int b = threadIdx.x; b < kBins; b += PH_THREADS) sh[b] = 0;
   __syncthreads();
   const float* src = raw + (size_t)g * T + rq.cu;
   float* dst = fresh + (size_t)g * T + rq.cu;
-  const int j0 = ch.key0 + (int)threadIdx.x * PH_PER;
-  float out[PH_PER];
-  if (!do_pool) {
+  const int t0 = (int)blockIdx.x * rq.span, t1 = min(rq.N, t0 + rq.span);
+  for (int j0 = t0 + (int)threadIdx.x * PH_PER; j0 < t1; j0 += PH_THREADS * PH_PER) {
+    float out[PH_PER];
+    if (!do_pool) {
 #pragma unroll
-    for (int e = 0; e < PH_PER; ++e) out[e] = j0 + e < rq.n ? dst[j0 + e] : CUDART_INF_F;
-  } else if (R >= 0) {
-    const float pad = mode == CAKE_POOL_MAX ? -CUDART_INF_F : 0.f;
-    float w[PH_PER + 2 * (R >= 0 ? R : 0)];
+      for (int e = 0; e < PH_PER; ++e) out[e] = j0 + e < rq.n ? dst[j0 + e] : CUDART_INF_F;
+    } else if (R >= 0) {
+      const float pad = mode == CAKE_POOL_MAX ? -CUDART_INF_F : 0.f;
+      float w[PH_PER + 2 * (R >= 0 ? R : 0)];
 #pragma unroll
-    for (int x = 0; x < PH_PER + 2 * R; ++x) {
-      const int j = j0 - R + x;
-      w[x] = (j >= 0 && j < rq.n) ? src[j] : pad;
-    }
+      for (int x = 0; x < PH_PER + 2 * R; ++x) {
+        const int j = j0 - R + x;
+        w[x] = (j >= 0 && j < rq.n) ? src[j] : pad;
+      }
 #pragma unroll
-    for (int e = 0; e < PH_PER; ++e) {
-      float m = w[e];
+      for (int e = 0; e < PH_PER; ++e) {
+        float m = w[e];
 #pragma unroll
-      for (int x = 1; x <= 2 * R; ++x) m = mode == CAKE_POOL_MAX ? fmaxf(m, w[e + x]) : m + w[e + x];
-      out[e] = mode == CAKE_POOL_MAX ? m : m / (float)kp;
-    }
-  } else {
-    const int r = kp >> 1;
+        for (int x = 1; x <= 2 * R; ++x) m = mode == CAKE_POOL_MAX ? fmaxf(m, w[e + x]) : m + w[e + x];
+        out[e] = mode == CAKE_POOL_MAX ? m : m / (float)kp;
+      }
+    } else {
+      const int r = kp >> 1;
 #pragma unroll 1
+      for (int e = 0; e < PH_PER; ++e) {
+        const int j = j0 + e;
+        float m = 0.f;
+        if (j < rq.n) {
+          const int a = max(0, j - r), b = min(rq.n, j + r + 1);
+          m = src[a];
+          for (int x = a + 1; x < b; ++x) m = mode == CAKE_POOL_MAX ? fmaxf(m, src[x]) : m + src[x];
+          if (mode != CAKE_POOL_MAX) m /= (float)kp;
+        }
+        out[e] = m;
+      }
+    }
+    // write back and count buckets; neighbours often share a bucket, so runs are counted once
+    int run_bin = -1;
+    uint32_t run_len = 0;
+#pragma unroll
     for (int e = 0; e < PH_PER; ++e) {
       const int j = j0 + e;
-      float m = 0.f;
-      if (j < rq.n) {
-        const int a = max(0, j - r), b = min(rq.n, j + r + 1);
-        m = src[a];
-        for (int x = a + 1; x < b; ++x) m = mode == CAKE_POOL_MAX ? fmaxf(m, src[x]) : m + src[x];
-        if (mode != CAKE_POOL_MAX) m /= (float)kp;
-      }
-      out[e] = m;
-    }
-  }
-  // write back and count buckets; neighbours often share a bucket, so runs are counted once
-  int run_bin = -1;
-  uint32_t run_len = 0;
-#pragma unroll
-  for (int e = 0; e < PH_PER; ++e) {
-    const int j = j0 + e;
-    if (j < ch.key0 + ch.nkeys) {
-      if (j >= rq.n) {
-        dst[j] = CUDART_INF_F;
-      } else {
-        if (do_pool) dst[j] = out[e];
-        const int q = bucket_of(ordered_key(out[e]));
-        if (q != run_bin) {
-          if (run_len) atomicAdd(&sh[run_bin], run_len);
-          run_bin = q;
-          run_len = 0;
+      if (j < t1) {
+        if (j >= rq.n) {
+          dst[j] = CUDART_INF_F;
+        } else {
+          if (do_pool) dst[j] = out[e];
+          const int q = bucket_of(ordered_key(out[e]));
+          if (q != run_bin) {
+            if (run_len) atomicAdd(&sh[run_bin], run_len);
+            run_bin = q;
+            run_len = 0;
+          }
+          ++run_len;
         }
-        ++run_len;
       }
     }
+    if (run_len) atomicAdd(&sh[run_bin], run_len);
   }
-  if (run_len) atomicAdd(&sh[run_bin], run_len);
   __syncthreads();
   uint32_t* gh = hist + (size_t)pair * kBins;
   for (int b = threadIdx.x; b < kBins; b += PH_THREADS)
@@ -264,13 +266,13 @@ pool_hist(const float* __restrict__ raw, float* __restrict__ fresh, const ReqInf
   __syncthreads();
   if (threadIdx.x == 0) {
     const uint32_t old = atomicAdd(&arrivals[pair], 1u);
-    s_last = (old + 1u == (uint32_t)rq.nchunks) ? 1 : 0;
+    s_last = (old + 1u == (uint32_t)rq.nsplit) ? 1 : 0;
   }
   __syncthreads();
   if (!s_last) return;
   __threadfence();
   // bucket offsets of the new list: prefix[i] = elements in buckets before i
-  int32_t* pf = prefix + (((size_t)ch.req * L + layer) * Hkv + g) * (kBins + 1);
+  int32_t* pf = prefix + (((size_t)req * L + layer) * Hkv + g) * (kBins + 1);
   constexpr int PER = kBins / PH_THREADS;
   int cnt[PER], sum = 0;
 #pragma unroll
@@ -499,16 +501,28 @@ __device__ inline void radix_digit(const uint2* __restrict__ e, int cnt, uint32_
 
 // Moves the threshold of one list to the budget b: the retained set becomes the first b entries
 // in the order (indicator descending, position ascending)  (Section 4.2 EVICT, Eq. 12).
+// `hint` >= 0 is the list's previous threshold bucket: budgets only shrink, so the new one is
+// that bucket or one shortly before it.
 __device__ void set_threshold(const int32_t* __restrict__ pf, const uint2* __restrict__ list, int b,
-                              ListState* __restrict__ out, EvictSmem& S) {
+                              int hint, ListState* __restrict__ out, EvictSmem& S) {
   if (b <= 0) {
     if (threadIdx.x == 0) *out = ListState{-1, 0xFFFFFFFFu, -1, 0};
     return;
   }
   // threshold bucket d: first bucket with prefix[d+1] >= b
-  int less = 0;
-  for (int i = threadIdx.x; i < kBins; i += blockDim.x) less += __ldcg(&pf[i + 1]) < b ? 1 : 0;
-  block_excl_scan(less, S.warp_tot, &S.total);
+  if (threadIdx.x == 0) S.total = -1;
+  __syncthreads();
+  if (hint >= 0) {
+    const int q = hint - (int)threadIdx.x;
+    if (q >= 0 && __ldcg(&pf[q]) < b && __ldcg(&pf[q + 1]) >= b) S.total = q;
+  }
+  __syncthreads();
+  if (S.total < 0) {
+    __syncthreads();
+    int less = 0;
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) less += __ldcg(&pf[i + 1]) < b ? 1 : 0;
+    block_excl_scan(less, S.warp_tot, &S.total);
+  }
   const int d = S.total;
   __syncthreads();
   if (d >= kBins) {                                  // b exceeds the stored entries: keep all
@@ -582,79 +596,57 @@ struct EvictArgs {
   uint32_t* fill;          // [pairs][kBins], zero between launches
   uint32_t* arrivals;      // [pairs]
   const ReqInfo* reqs;
-  const ScoreUnit* chunks;
   const int32_t* cur;      // budgets of this stage
-  int n_chunks, stage, L, Hkv, n_req;
+  int stage, L, Hkv;
   int64_t T;
 };
 
-// Stage `stage` of the cascade.  CTAs [0, n_chunks * Hkv): scatter one chunk of the newest
-// layer's pooled indicators into bucket order (only the buckets its budget can ever reach; the
-// budget never grows again, Proposition 1); the CTA that completes a list sets its threshold.
-// The remaining CTAs move the threshold of one older list each to its new budget.
-__global__ void __launch_bounds__(EV_THREADS)
-evict_stage(const EvictArgs A) {
+constexpr int SC_THREADS = 1024;
+constexpr int SC_PER = 4;
+
+// Newest layer of stage `stage`: one CTA per (split of a request's tokens, KV head, request)
+// scatters the pooled indicators into bucket order.  Only the buckets the layer's budget can
+// ever reach are stored (the budget never grows again, Proposition 1).  The CTA that completes
+// a list sets its threshold.
+__global__ void __launch_bounds__(SC_THREADS)
+scatter_new(const EvictArgs A) {
   __shared__ EvictSmem S;
   __shared__ uint32_t s_cnt[kBins];
   __shared__ uint32_t s_base[kBins];
   __shared__ int s_last;
-  const int n_scatter = A.n_chunks * A.Hkv;
-  if ((int)blockIdx.x >= n_scatter) {
-    // ---- older list: (request, layer < stage, head)
-    int idx = (int)blockIdx.x - n_scatter;
-    const int g = idx % A.Hkv; idx /= A.Hkv;
-    const int layer = idx % A.stage;
-    const int req = idx / A.stage;
-    const ReqInfo rq = A.reqs[req];
-    const size_t lid = ((size_t)req * A.L + layer) * A.Hkv + g;
-    const int b = min(A.cur[(size_t)req * A.L + layer], rq.n);
-    if (A.states[lid].kept == b) return;                       // budget unchanged
-    set_threshold(A.prefix_all + lid * (kBins + 1),
-                  A.lists + rq.list_off + ((size_t)layer * A.Hkv + g) * rq.n, b, &A.states[lid], S);
-    return;
-  }
-  // ---- newest layer: scatter chunk
-  const ScoreUnit ch = A.chunks[blockIdx.x / A.Hkv];
-  const int g = blockIdx.x % A.Hkv;
-  const ReqInfo rq = A.reqs[ch.req];
-  const int pair = ch.req * A.Hkv + g;
-  const size_t lid = ((size_t)ch.req * A.L + A.stage) * A.Hkv + g;
+  const int g = blockIdx.y, req = blockIdx.z;
+  const ReqInfo rq = A.reqs[req];
+  if ((int)blockIdx.x >= rq.nsplit) return;
+  const int pair = req * A.Hkv + g;
+  const size_t lid = ((size_t)req * A.L + A.stage) * A.Hkv + g;
   const int32_t* pf = A.prefix_all + lid * (kBins + 1);
   uint2* list = A.lists + rq.list_off + ((size_t)A.stage * A.Hkv + g) * rq.n;
-  const int b = min(A.cur[(size_t)ch.req * A.L + A.stage], rq.n);
+  const int b = min(A.cur[(size_t)req * A.L + A.stage], rq.n);
   // last bucket worth storing
   int less = 0;
-  for (int i = threadIdx.x; i < kBins; i += EV_THREADS) {
+  for (int i = threadIdx.x; i < kBins; i += SC_THREADS) {
     less += __ldcg(&pf[i + 1]) < b ? 1 : 0;
     s_cnt[i] = 0;
   }
   block_excl_scan(less, S.warp_tot, &S.total);
   const int d_last = b > 0 ? min(S.total, kBins - 1) : -1;
   __syncthreads();
-  // a thread owns PER consecutive tokens; runs of equal buckets are counted and placed at once
-  constexpr int PER = kChunkKeys / EV_THREADS;
-  uint32_t key[PER];
-  int bk[PER];
   const float* src = A.fresh + (size_t)g * A.T + rq.cu;
-  const int j0 = ch.key0 + (int)threadIdx.x * PER;
-#pragma unroll
-  for (int e = 0; e < PER; ++e) {
-    const int j = j0 + e;
-    bk[e] = -1;
-    if (j < rq.n && j < ch.key0 + ch.nkeys) {
-      key[e] = ordered_key(src[j]);
-      const int q = bucket_of(key[e]);
-      if (q <= d_last) bk[e] = q;
-    }
-  }
-  {
+  const int t0 = (int)blockIdx.x * rq.span, t1 = min(rq.n, t0 + rq.span);
+  // pass 1: count this split's entries per bucket (runs of equal buckets at once)
+  for (int j0 = t0 + (int)threadIdx.x * SC_PER; j0 < t1; j0 += SC_THREADS * SC_PER) {
     int run_bin = -1;
     uint32_t run_len = 0;
 #pragma unroll
-    for (int e = 0; e < PER; ++e) {
-      if (bk[e] != run_bin) {
+    for (int e = 0; e < SC_PER; ++e) {
+      int q = -1;
+      if (j0 + e < t1) {
+        q = bucket_of(ordered_key(src[j0 + e]));
+        if (q > d_last) q = -1;
+      }
+      if (q != run_bin) {
         if (run_len && run_bin >= 0) atomicAdd(&s_cnt[run_bin], run_len);
-        run_bin = bk[e];
+        run_bin = q;
         run_len = 0;
       }
       ++run_len;
@@ -662,24 +654,37 @@ evict_stage(const EvictArgs A) {
     if (run_len && run_bin >= 0) atomicAdd(&s_cnt[run_bin], run_len);
   }
   __syncthreads();
+  // reserve this split's range inside every bucket of the list
   uint32_t* gf = A.fill + (size_t)pair * kBins;
-  for (int q = threadIdx.x; q < kBins; q += EV_THREADS) {
+  for (int q = threadIdx.x; q < kBins; q += SC_THREADS) {
     const uint32_t c = s_cnt[q];
     if (c) s_base[q] = (uint32_t)__ldcg(&pf[q]) + atomicAdd(&gf[q], c);
     s_cnt[q] = 0;
   }
   __syncthreads();
-  {
+  // pass 2: place the entries
+  for (int j0 = t0 + (int)threadIdx.x * SC_PER; j0 < t1; j0 += SC_THREADS * SC_PER) {
+    uint32_t key[SC_PER];
+    int bk[SC_PER];
+#pragma unroll
+    for (int e = 0; e < SC_PER; ++e) {
+      bk[e] = -1;
+      if (j0 + e < t1) {
+        key[e] = ordered_key(src[j0 + e]);
+        const int q = bucket_of(key[e]);
+        if (q <= d_last) bk[e] = q;
+      }
+    }
     int run_bin = -1;
     uint32_t run_off = 0;
 #pragma unroll
-    for (int e = 0; e < PER; ++e) {
+    for (int e = 0; e < SC_PER; ++e) {
       if (bk[e] != run_bin) {
         run_bin = bk[e];
         if (run_bin >= 0) {
           uint32_t len = 1;
 #pragma unroll
-          for (int f = e + 1; f < PER; ++f) {
+          for (int f = e + 1; f < SC_PER; ++f) {
             if (bk[f] != run_bin) break;
             ++len;
           }
@@ -693,14 +698,30 @@ evict_stage(const EvictArgs A) {
   __syncthreads();
   if (threadIdx.x == 0) {
     const uint32_t old = atomicAdd(&A.arrivals[pair], 1u);
-    s_last = (old + 1u == (uint32_t)rq.nchunks) ? 1 : 0;
+    s_last = (old + 1u == (uint32_t)rq.nsplit) ? 1 : 0;
   }
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  for (int q = threadIdx.x; q < kBins; q += EV_THREADS) gf[q] = 0;       // ready for the next stage
+  for (int q = threadIdx.x; q < kBins; q += SC_THREADS) gf[q] = 0;       // ready for the next stage
   if (threadIdx.x == 0) A.arrivals[pair] = 0;
-  set_threshold(pf, list, b, &A.states[lid], S);
+  set_threshold(pf, list, b, -1, &A.states[lid], S);
+}
+
+// Older layers of stage `stage`: one CTA per (KV head, layer < stage, request) moves the list's
+// threshold to its new budget.
+__global__ void __launch_bounds__(EV_THREADS)
+thresholds_old(const EvictArgs A) {
+  __shared__ EvictSmem S;
+  const int g = blockIdx.x, layer = blockIdx.y, req = blockIdx.z;
+  const ReqInfo rq = A.reqs[req];
+  const size_t lid = ((size_t)req * A.L + layer) * A.Hkv + g;
+  const int b = min(A.cur[(size_t)req * A.L + layer], rq.n);
+  const ListState old = A.states[lid];
+  if (old.kept == b) return;                                   // budget unchanged
+  set_threshold(A.prefix_all + lid * (kBins + 1),
+                A.lists + rq.list_off + ((size_t)layer * A.Hkv + g) * rq.n, b, old.bucket,
+                &A.states[lid], S);
 }
 
 }  // namespace
@@ -728,19 +749,18 @@ int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, bool finalize, c
     F.fin_arrivals = ctx->d_arrivals + ctx->max_pairs;
     F.dH = ctx->d_H; F.dV = ctx->d_V; F.dP = ctx->d_P;
     F.status = ctx->d_status;
-    F.units = ctx->n_req * (c.n_q_heads / c.n_kv_heads);
+    F.units = c.n_q_heads / c.n_kv_heads;
     F.use_hrow = ctx->hhead_from_rows ? 1 : 0;
     F.rows = ctx->rows;
     F.inv_tau1 = 1.0 / (double)c.tau1;
     F.inv_tau2 = 1.0 / (double)c.tau2;
   }
-  if (ctx->n_chunks + F.units == 0) return cuda_status(cudaGetLastError());
-  const dim3 grid((unsigned)(ctx->n_chunks + F.units), c.n_kv_heads);
+  const dim3 grid((unsigned)(ctx->n_split + F.units), c.n_kv_heads, ctx->n_req);
   const int r = c.pool_kernel / 2;
 #define CAKE_POOL_LAUNCH(RR)                                                                     \
-  pool_hist<RR><<<grid, PH_THREADS, 0, st>>>(ctx->d_raw[layer & 1], ctx->d_fresh, ctx->d_req, ctx->d_chunks, \
+  pool_hist<RR><<<grid, PH_THREADS, 0, st>>>(ctx->d_raw[layer & 1], ctx->d_fresh, ctx->d_req,    \
                                              ctx->d_hist, ctx->d_arrivals, ctx->d_prefix,        \
-                                             ctx->n_chunks, layer, c.n_layers, c.n_kv_heads,     \
+                                             ctx->n_split, layer, c.n_layers, c.n_kv_heads,      \
                                              ctx->total_tokens, c.pool_kernel, c.pool_mode,      \
                                              do_pool ? 1 : 0, F)
   switch (r) {
@@ -776,14 +796,14 @@ int32_t launch_evict(cake_ctx* ctx, int32_t stage, cudaStream_t st) {
   A.fill = ctx->d_fill;
   A.arrivals = ctx->d_arrivals;
   A.reqs = ctx->d_req;
-  A.chunks = ctx->d_chunks;
   A.cur = ctx->d_budget[stage & 1];
-  A.n_chunks = ctx->n_chunks; A.stage = stage; A.L = c.n_layers; A.Hkv = c.n_kv_heads;
-  A.n_req = ctx->n_req;
+  A.stage = stage; A.L = c.n_layers; A.Hkv = c.n_kv_heads;
   A.T = ctx->total_tokens;
-  const unsigned grid = (unsigned)(ctx->n_chunks * c.n_kv_heads + stage * c.n_kv_heads * ctx->n_req);
-  if (grid == 0) return CAKE_OK;
-  evict_stage<<<grid, EV_THREADS, 0, st>>>(A);
+  if (stage > 0) {
+    thresholds_old<<<dim3(c.n_kv_heads, stage, ctx->n_req), EV_THREADS, 0, st>>>(A);
+    count_launch();
+  }
+  scatter_new<<<dim3(ctx->n_split, c.n_kv_heads, ctx->n_req), SC_THREADS, 0, st>>>(A);
   count_launch();
   return cuda_status(cudaGetLastError());
 }
