@@ -68,8 +68,10 @@ __device__ inline double warp_sum_f64(double v) {
 // scattered into bucket order by the eviction kernel; from then on "keep the top b" means
 // "all buckets before the one that contains the b-th element, plus the best part of that
 // bucket", so a later, smaller budget only moves a threshold and rewrites nothing.
+// Order-preserving integer image of a float; -0 and +0 compare equal, as they do as floats.
 __device__ inline uint32_t ordered_key(float v) {
-  const uint32_t b = __float_as_uint(v);
+  uint32_t b = __float_as_uint(v);
+  if (b == 0x80000000u) b = 0u;
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 __device__ inline int bucket_of(uint32_t key) { return (kBins - 1) - (int)(key >> (32 - kBinBits)); }

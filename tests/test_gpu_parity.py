@@ -347,6 +347,26 @@ def test_selection_with_massive_ties_and_negative_values():
     cake.destroy()
 
 
+def test_negative_zero_ties_with_positive_zero():
+    """-0.0 and +0.0 are equal indicators: the lower position wins, as in the oracle."""
+    w = small_w(n_layers=1, seq_lens=(400,), total_budget=16 + 100)
+    T = w.total_tokens
+    ind = np.full((w.n_kv_heads, T), -1.0, dtype=np.float32)
+    ind[:, 0:300:2] = 0.0
+    ind[:, 1:300:2] = -0.0
+    ind[:, 350:360] = 1.0
+    P = np.array([[1.0]])
+    cake = harness.cake_for(w)
+    run_cascade_on(cake, w, [torch.from_numpy(ind).cuda()], P)
+    b = cake.get_budgets().cpu().numpy()
+    c = O.cascade([ind[:, :T - 16].astype(np.float64)], P[0], total_budget=w.total_budget,
+                  window=16, seq_len=T)
+    got = cake.get_positions(0, 0, int(b[0, 0])).cpu().numpy()
+    for g in range(w.n_kv_heads):
+        assert np.array_equal(got[g], c.positions[0][g])
+    cake.destroy()
+
+
 def test_empty_batch_and_call_order_errors():
     w = small_w()
     cake = harness.cake_for(w)
