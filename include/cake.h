@@ -187,6 +187,31 @@ int32_t cake_profile_read(cake_ctx* ctx, double* ms_out, int64_t* spans_out, voi
  * SIMT kernels, negative on error. */
 int32_t cake_uses_tensor_cores(const cake_ctx* ctx);
 
+/* ---- selection without any allocation ------------------------------------- */
+/* The paper has no counterpart for this entry point; it exists for callers that are not
+ * allowed to allocate device memory when they call in: code running inside another
+ * framework's memory pool or a fixed memory plan, a real-time or serving loop where
+ * cudaMalloc / cudaFree would stall the device, or a process whose allocator is already
+ * exhausted on purpose.  Such callers cannot use a context (cake_create allocates).
+ *
+ * Per head, keeps the `keep` entries of values[head][0..n) that come first in the order
+ * (value descending, position ascending) -- the TopK of Eq. 12 with the same tie rule as
+ * cake_evict -- and writes their positions in ascending order.
+ *   values        device fp32 [n_heads][n]
+ *   positions_out device int32 [n_heads][keep]
+ * It calls no cudaMalloc, cudaFree or other allocating routine.  Its working memory (two
+ * bitmaps per head) is a fixed 256 KB array inside the library, present on every GPU that
+ * loads the library until the process exits, which bounds the problem size:
+ *   n_heads * ceil(n / 32) <= 32768      (about one million values per call);
+ * anything larger returns CAKE_ERR_CAPACITY and does nothing.  0 <= keep <= n, else
+ * CAKE_ERR_ARG.  All calls share that array and the array keeps the previous call's
+ * contents; the kernel clears what it needs first, but two calls that overlap on the GPU
+ * (different streams, or different host threads without ordering) race on it: serialise them.
+ * The first call on each device looks up the array's device address (once per device, with
+ * that device current); make that first call outside any stream capture. */
+int32_t cake_select_positions_static(const float* values, int32_t n_heads, int32_t n, int32_t keep,
+                                     int32_t* positions_out, void* stream);
+
 const char* cake_strerror(int32_t code);
 /* Number of kernels this library has launched in the calling process. */
 int64_t cake_launch_count(void);

@@ -29,6 +29,7 @@ EXPORTS = [
     "cake_get_preferences", "cake_get_budgets", "cake_get_positions", "cake_set_indicators",
     "cake_set_preferences", "cake_status", "cake_strerror", "cake_launch_count",
     "cake_profile_enable", "cake_profile_read", "cake_uses_tensor_cores",
+    "cake_select_positions_static",
 ]
 PROF_KINDS = ["score", "finalize", "allocate", "evict", "compact"]
 
@@ -84,6 +85,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.cake_profile_enable.argtypes = [vp, i32]
     lib.cake_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64), vp]
     lib.cake_uses_tensor_cores.argtypes = [vp]
+    lib.cake_select_positions_static.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.cake_strerror.argtypes = [i32]
     lib.cake_strerror.restype = ctypes.c_char_p
     lib.cake_launch_count.argtypes = []
@@ -123,6 +125,21 @@ def _ptr(t: Optional[torch.Tensor], dtype: Optional[torch.dtype] = None) -> Opti
 
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
+
+
+def select_positions_static(values: torch.Tensor, keep: int,
+                            out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """cake_select_positions_static: per-head top-`keep` positions (ascending) of a CUDA fp32
+    tensor [n_heads][n], for callers that may not allocate device memory.  The library call
+    allocates nothing; pass `out` (int32 [n_heads][keep]) to keep torch from allocating too."""
+    n_heads, n = values.shape
+    if out is None:
+        out = torch.empty(n_heads, max(keep, 1), dtype=torch.int32, device=values.device)[:, :keep]
+        out = out.contiguous()
+    _check(load_library().cake_select_positions_static(
+        _ptr(values, torch.float32), n_heads, n, keep, _ptr(out, torch.int32) if keep > 0 else None,
+        _stream()), "cake_select_positions_static")
+    return out
 
 
 class Cake:

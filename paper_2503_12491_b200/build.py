@@ -16,7 +16,8 @@ CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG, "libcake.so")
 
-SOURCES = ["cake_api.cu", "score_simt.cu", "score_tc.cu", "cascade.cu", "compact.cu"]
+SOURCES = ["cake_api.cu", "score_simt.cu", "score_tc.cu", "cascade.cu", "compact.cu",
+           "select_static.cu"]
 
 
 def _nvcc() -> str:
