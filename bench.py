@@ -166,6 +166,22 @@ def workload_config(w):
             "parallelism": "replicas only"}
 
 
+# ------------------------------------------------------------- replicas
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time: replicas do not exchange data, only this number."""
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_rank: int, world: int, ms_step: float) -> float:
+    """Whole-job throughput of `world` independent replicas that all finish within ms_step."""
+    return tokens_per_rank * world / (ms_step * 1e-3)
+
+
 # --------------------------------------------------------------- CUDA leg
 def main():
     args = parse_args()
@@ -254,12 +270,8 @@ def main():
     ms_profiled = evp0.elapsed_time(evp1) / args.steps
     cake.profile_enable(False)
     clocks = sampler.stop() if rank == 0 else None
-    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
-    tokens = w.total_tokens * world
-    value = tokens / (ms_step * 1e-3)
+    ms_step = max_over_ranks(ms_total, world, "cuda") / args.steps
+    value = whole_job_value(w.total_tokens, world, ms_step)
 
     retained_rows = int(bufs[2][-1].item())
     k_bytes = L * w.n_kv_heads * w.total_tokens * w.head_dim * esize
@@ -360,11 +372,7 @@ def e2e_leg(args, w, cake, qs, ks, vs, bufs, world, barrier):
     ev1.record()
     barrier()
     ms = ev0.elapsed_time(ev1) / steps
-    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms = float(t.item())
+    ms = max_over_ranks(ms, world, "cuda")
     esize = 4 if w.dtype == "fp32" else 2
     h2d = sum(x.numel() * x.element_size() for x in hq + hk + hv)
     d2h = 2 * n * w.head_dim * esize + n * 4 + out_off.numel() * 8

@@ -16,8 +16,19 @@
  *     the caller owns and keeps alive until the stream has consumed them.  The
  *     context owns only its own state and scratch (allocated in cake_create).
  *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work;
- *     none synchronises with the device except cake_status, cake_destroy and
- *     the *_host convenience entry points, which say so.
+ *     none synchronises the host with the device except cake_status,
+ *     cake_profile_read and cake_destroy, which say so.
+ *   - Stream order.  cake_score_layer runs on the caller's stream.  Everything
+ *     that follows a layer's scoring (pooling, preference, cake_allocate,
+ *     cake_evict) is enqueued on a stream the context owns, ordered after that
+ *     layer's score kernel by events, so that it runs beside the scoring of the
+ *     next layer.  cake_compact, every cake_get_* / cake_set_* call, cake_begin
+ *     and cake_status first make the stream they are given wait for that
+ *     internal work.  Hence: results are ordered into the caller's stream by
+ *     the call that hands them out, not by cake_allocate / cake_evict
+ *     themselves, and the stream arguments of those two calls are unused.
+ *     Q and K of a layer are read only by cake_score_layer's kernels (caller's
+ *     stream); K and V are read again by cake_compact.
  *   - A context serves one batch of requests at a time and is not thread-safe.
  *
  * Shapes: L layers, H_q query heads, H_kv KV heads, G = H_q/H_kv, d = head_dim,
@@ -119,7 +130,11 @@ int32_t cake_allocate(cake_ctx* ctx, int32_t stage, void* stream);
  * come first in the order (indicator descending, token position ascending)
  * among the stored (indicator, position) pairs; survivors keep their stored
  * indicator.  The window tokens are always kept.  Needs cake_allocate(stage)
- * and stages in order. */
+ * and stages in order.
+ * The stored pairs of a layer are kept sorted by the leading bits of the
+ * indicator (written once, when the layer arrives); a later, smaller budget
+ * only moves the list's threshold, which selects the same set as a TopK on the
+ * surviving pairs would. */
 int32_t cake_evict(cake_ctx* ctx, int32_t stage, void* stream);
 
 /* Gathers the retained rows of layers [layer_lo, layer_hi) (Eq. 12: K^ = K[D,:],

@@ -229,6 +229,47 @@ def test_end_to_end_own_indicators_differ_only_near_threshold(case):
     cake.destroy()
 
 
+# ------------------------------------------------ full size, as the benchmark launches it
+def test_one_full_size_layer_of_the_128k_workload():
+    """Layer 0 of the 128K Llama-3.1-8B-shaped workload at full length, in the launch
+    configuration the benchmark times (same context geometry; only the layer count and the
+    budget are scaled to one layer): every indicator and H, V, P against the oracle, then the
+    selection on the device's own indicators, and the planted needles."""
+    full = synth.workload(4)
+    w = synth.scaled(full, n_layers=1, total_budget=full.total_budget // full.n_layers)
+    qs, ks, vs = harness.device_inputs(w)
+    cake = harness.cake_for(w)
+    k_out, v_out, off, pos = cake.run(qs, ks, vs, w.cu_seqlens)
+    assert cake.status() == 0
+    N = w.seq_lens[0]
+    n = N - w.window
+    ref = O.score_layer(to_np(qs[0][0]), to_np(ks[0]), gamma=w.gamma, pool_kernel=w.pool_kernel,
+                        tau1=w.tau1, tau2=w.tau2)
+    ind = cake.get_indicators(0).cpu().numpy()
+    assert_close(ind[:, :n], ref["indicator"], "indicator at 128K")
+    H, V, P = (x.cpu().numpy() for x in cake.get_preferences())
+    assert_close(H[0, 0], ref["H"], "H at 128K")
+    assert_close(V[0, 0], ref["V"], "V at 128K")
+    assert_close(P[0, 0], ref["P"], "P at 128K")
+    b = int(cake.get_budgets().cpu().numpy()[0, 0]) - w.window
+    assert b == w.total_budget - w.window
+    got = harness.split_blocks(w, pos, off)[0][0].cpu().numpy()
+    needles = np.array(synth.needle_positions(w, 0))
+    for g in range(w.n_kv_heads):
+        assert np.all(np.diff(got[g]) > 0) and np.array_equal(got[g][b:], np.arange(n, N))
+        want = O.topk_keep(ref["indicator"][g], b)
+        diff = np.setxor1d(got[g][:b], want)
+        if diff.size:
+            thr = np.sort(ref["indicator"][g])[::-1][b - 1]
+            rel = np.abs(ref["indicator"][g][diff] - thr) / thr
+            assert rel.max() <= 2 * RTOL, (g, diff.size, rel.max())
+        if np.isin(needles, want).all():              # the oracle keeps every needle: so must we
+            assert np.isin(needles, got[g][:b]).all(), g
+        src = ks[0][g, torch.from_numpy(got[g]).long().cuda()]
+        assert torch.equal(harness.split_blocks(w, k_out, off)[0][0][g], src)
+    cake.destroy()
+
+
 # ---------------------------------------------------------------- edge cases
 def small_w(**kw):
     base = synth.scaled(synth.workload(1), n_layers=2, seq_lens=(100,), total_budget=2 * 30)
