@@ -24,6 +24,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "CAKE score+evict+compact prompt tokens/s"
+# DRAM bytes of one score-kernel launch at workload 4 from the ncu capture under profiles/;
+# set to None whenever the kernel changes until the counters are taken again.
+SCORE_KERNEL_DRAM_BYTES = 271670528 + 9626112
 UNIT = "tokens/s"
 
 
@@ -289,7 +292,11 @@ def main():
     step_gbps = ideal / (ms_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak,
                 "unit": "GB/s", "frac": (achieved / hbm_peak) if achieved else None,
-                "peak_kind": f"{peak_kind} copy bandwidth", "traffic": None,
+                "peak_kind": f"{peak_kind} copy bandwidth",
+                "traffic": SCORE_KERNEL_DRAM_BYTES if args.workload == 4 else None,
+                "traffic_source": "profiles/score_fused_kernel_llama31-8b-gqa-128k_2layers.md "
+                                  "(dram__bytes_read.sum + dram__bytes_write.sum of one launch; a "
+                                  "launch of the reduced case is a full-size launch)",
                 "bytes_per_launch": per_launch_bytes, "ms_per_launch": dom_ms,
                 "launches_timed": prof[dom]["spans"],
                 "phase_ms_per_step": phase_ms, "ms_per_step_with_brackets": ms_profiled,
