@@ -56,6 +56,7 @@ constexpr long long kSpinLimit = 4000000000ll;   // cycles (~2 s) before a wait 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLazyMax = 8.f;      // pass A rescales only when the row max grows by 2^8
 constexpr int64_t kWaveBytes = 32ll << 20;
+constexpr int kWaveDepth = 1;         // pass B of a wave follows pass A of the wave this far ahead
 
 struct TcParams {
   const ScoreOp* ops;
@@ -837,7 +838,8 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
     wave_begin.push_back(n_pairs);
   }
   const int n_waves = (int)wave_begin.size() - 1;
-  std::vector<std::vector<ScoreOp>> full(n_cta), bonly(n_cta), wa(n_cta), wb(n_cta), wb_prev(n_cta);
+  std::vector<std::vector<ScoreOp>> full(n_cta), bonly(n_cta), wa(n_cta), wb(n_cta);
+  std::vector<std::vector<std::vector<ScoreOp>>> wbs;      // pass-B ops of every wave, per CTA
   int32_t aseg = 0, bseg = 0;
   int32_t* pair_aseg = ctx->h_tc_index;                    // [pairs+1]
   int32_t* pair_bseg = ctx->h_tc_index + (n_pairs + 1);    // [pairs+1]
@@ -862,15 +864,19 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
     }
     // a wave's remainder tiles land on different CTAs each time (golden-ratio stride)
     rot = (rot + (int)(n_cta * 0.381966) + 1) % n_cta;
+    wbs.push_back(wb);
     for (int cta = 0; cta < n_cta; ++cta) {
       full[cta].insert(full[cta].end(), wa[cta].begin(), wa[cta].end());
-      if (wv > 0) full[cta].insert(full[cta].end(), wb_prev[cta].begin(), wb_prev[cta].end());
+      if (wv >= kWaveDepth) {
+        const std::vector<ScoreOp>& due = wbs[wv - kWaveDepth][cta];
+        full[cta].insert(full[cta].end(), due.begin(), due.end());
+      }
       bonly[cta].insert(bonly[cta].end(), wb[cta].begin(), wb[cta].end());
     }
-    wb_prev.swap(wb);
   }
-  for (int cta = 0; cta < n_cta; ++cta)
-    full[cta].insert(full[cta].end(), wb_prev[cta].begin(), wb_prev[cta].end());
+  for (int wv = n_waves > kWaveDepth ? n_waves - kWaveDepth : 0; wv < n_waves; ++wv)
+    for (int cta = 0; cta < n_cta; ++cta)
+      full[cta].insert(full[cta].end(), wbs[wv][cta].begin(), wbs[wv][cta].end());
   pair_aseg[n_pairs] = aseg;
   pair_bseg[n_pairs] = bseg;
   if (aseg > ctx->max_tc_segs || bseg > ctx->max_tc_segs) return CAKE_ERR_CAPACITY;
