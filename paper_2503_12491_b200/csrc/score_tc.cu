@@ -440,7 +440,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     }
   } else if (warp == WARP_MERGE) {
     // ------------------------------------------------ row merger
-    // Row r of every pair is merged by CTA r % gridDim.x: once all partials of the pair have
+    // Every (pair, row) is merged by one CTA of the grid: once all partials of the pair have
     // been delivered, the warp loads the row's partials in one round trip, merges them in a
     // fixed order and publishes the row's base-2 log-sum-exp and entropy term.
     if (P.pair_done) {
@@ -448,7 +448,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       for (int pair = 0; pair < P.n_pairs && ok; ++pair) {
         const int s_lo = P.pair_aseg[pair] * NWG, s_hi = P.pair_aseg[pair + 1] * NWG;
         bool waited = false;
-        for (int r = blockIdx.x; r < P.rows; r += gridDim.x) {
+        // row r of pair p belongs to CTA (p * rows + r) % grid: with many short pairs every CTA
+        // gets a few (pair, row) items instead of the first `rows` CTAs getting all of them
+        const int r0 = (int)((blockIdx.x + gridDim.x - (unsigned)(((long long)pair * P.rows) % gridDim.x)) % gridDim.x);
+        for (int r = r0; r < P.rows; r += gridDim.x) {
           if (!waited) {
             const uint32_t want = (uint32_t)(s_hi - s_lo) * 4u * P.epoch;   // one per warp
             const long long t0 = clock64();
@@ -633,6 +636,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * 128);
           const int key0 = op.key0 + it * TILE;
           const bool interior = key0 + TILE <= op.n && it * TILE + TILE <= op.nkeys;
+          if (quad * 32 >= P.rows) {                   // these TMEM lanes hold padding rows
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.acc_empty[b]);
+            continue;
+          }
 #pragma unroll 1
           for (int c0 = 0; c0 < TILE; c0 += 32) {
             uint32_t r[32];
