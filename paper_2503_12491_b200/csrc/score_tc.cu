@@ -86,7 +86,8 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+  asm volatile("{\n.reg .pred e;\nelect.sync _|e, 0xffffffff;\n"
+               "@e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n}" ::"r"(smem_u32(bar)),
                "r"(bytes)
                : "memory");
 }
@@ -120,8 +121,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_
 __device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* map, uint64_t* bar,
                                                  int c0, int c1, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-      "[%0], [%1, {%3, %4}], [%2], %5;"
+      "{\n.reg .pred e;\nelect.sync _|e, 0xffffffff;\n"
+      "@e cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4}], [%2], %5;\n}"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "l"(policy)
       : "memory");
 }
@@ -138,7 +140,8 @@ __device__ __forceinline__ uint64_t l2_policy_evict_first() {
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0,
                                             int c1, int c2, int c3) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      "{\n.reg .pred e;\nelect.sync _|e, 0xffffffff;\n"
+      "@e cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n}"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
@@ -148,37 +151,41 @@ __device__ __forceinline__ void tc_fence_before() {
 __device__ __forceinline__ void tc_fence_after() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
-// The issuing thread is a single lane whose dependent instructions run at a few cycles each, so
-// the per-MMA work is kept minimal: descriptors differ only in the 14-bit address field of their
-// low word, the high word (stride, version, swizzle) is a constant, and the accumulate flag is
-// an immediate.
+// The MMA and TMA warps run converged, all 32 lanes executing the same loop, and one elected lane
+// issues each asynchronous instruction.  Issued from inside a one-lane branch the operands of
+// every tcgen05.mma are moved to uniform registers one by one and an M128 x N128 x K16 MMA costs
+// about 70 cycles to issue, more than the 64 cycles it takes to execute; from a converged warp
+// the descriptor arithmetic stays in the uniform datapath and the tensor pipe sets the pace.
+// Descriptors differ only in the 14-bit address field of their low word, the high word (stride,
+// version, swizzle) is a constant, and the accumulate flag is an immediate.
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // SBO, version 1, SWIZZLE_128B
 template <int kAcc>
 __device__ __forceinline__ void umma_ss(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
   asm volatile(
-      "{\n.reg .pred p;\n.reg .b64 da, db;\nsetp.ne.b32 p, %4, 0;\n"
+      "{\n.reg .pred p, e;\n.reg .b64 da, db;\nsetp.ne.b32 p, %4, 0;\nelect.sync _|e, 0xffffffff;\n"
       "mov.b64 da, {%1, %5};\nmov.b64 db, {%2, %5};\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n}"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n}"
       ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "n"(kAcc), "r"(kDescHi)
       : "memory");
 }
 template <int kAcc>
 __device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t idesc) {
   asm volatile(
-      "{\n.reg .pred p;\n.reg .b64 db;\nsetp.ne.b32 p, %4, 0;\n"
+      "{\n.reg .pred p, e;\n.reg .b64 db;\nsetp.ne.b32 p, %4, 0;\nelect.sync _|e, 0xffffffff;\n"
       "mov.b64 db, {%2, %5};\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n}"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n}"
       ::"r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(idesc), "n"(kAcc), "r"(kDescHi)
       : "memory");
 }
 // Copies 128 rows x 32 bytes (one K = 16 slice of a K-major operand) from shared to tensor memory.
 __device__ __forceinline__ void tmem_cp_128x256b(uint32_t tmem_dst, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(tmem_dst), "l"(sdesc) : "memory");
+  asm volatile("{\n.reg .pred e;\nelect.sync _|e, 0xffffffff;\n@e tcgen05.cp.cta_group::1.128x256b [%0], %1;\n}"
+               ::"r"(tmem_dst), "l"(sdesc) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                   smem_u32(bar))
-               : "memory");
+  asm volatile("{\n.reg .pred e;\nelect.sync _|e, 0xffffffff;\n"
+               "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}"
+               ::"r"(smem_u32(bar)) : "memory");
 }
 // Starts the load of 32 consecutive fp32 columns of this thread's TMEM lane; the registers
 // are valid only after tmem_ld_wait on the same array.
@@ -326,10 +333,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   const uint32_t tmem_base = *S.tmem_holder;
 
   if (warp == WARP_TMA) {
-    // ------------------------------------------------ TMA producer
-    if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&q_map) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
+    // ------------------------------------------------ TMA producer (converged warp, elected lane issues)
+    {
+      if (lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&q_map) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
+      }
+      __syncwarp();
       // pass A's tiles are read again by pass B: keep them in L2; pass B's read is the last
       const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
       uint32_t t = 0, qn = 0;
@@ -368,8 +378,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         mbar_wait(&S.q_full[u & 1], (u >> 1) & 1, P.status);
     }
   } else if (warp == WARP_MMA) {
-    // ------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------ MMA issuer (converged warp, elected lane issues)
+    {
       uint32_t t = 0, qn = 0;
       const uint32_t k_lo0 = (smem_u32(S.k) & 0x3FFFFu) >> 4;
       bool ok = true;
