@@ -2,6 +2,8 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <cstdio>
+#include <cstdlib>
 #include <cuda_bf16.h>
 #include <stdint.h>
 
@@ -188,12 +190,18 @@ int32_t launch_get_positions(cake_ctx* ctx, int32_t req, int32_t layer, int32_t*
 int prof_begin(cake_ctx* ctx, int kind, cudaStream_t st);
 void prof_end(cake_ctx* ctx, int span, cudaStream_t st);
 
-inline int32_t cuda_status(cudaError_t e) { return e == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA; }
+// Maps a CUDA runtime result to a library status; with CAKE_VERBOSE set in the environment the
+// runtime's own message goes to stderr, since the status code alone does not say which error it was.
+inline int32_t cuda_status(cudaError_t e) {
+  if (e == cudaSuccess) return CAKE_OK;
+  if (getenv("CAKE_VERBOSE")) fprintf(stderr, "libcake: CUDA error %d: %s\n", (int)e, cudaGetErrorString(e));
+  return CAKE_ERR_CUDA;
+}
 
 #define CAKE_CUDA_TRY(expr)                         \
   do {                                              \
     cudaError_t _e = (expr);                        \
-    if (_e != cudaSuccess) return CAKE_ERR_CUDA;    \
+    if (_e != cudaSuccess) return cuda_status(_e);  \
   } while (0)
 
 }  // namespace cake

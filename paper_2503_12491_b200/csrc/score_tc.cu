@@ -235,6 +235,17 @@ __device__ __forceinline__ void red_release_add(uint32_t* p, uint32_t v) {
   asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
+// A counter in shared memory that only grows: a wait for "at least v" cannot mistake one round
+// for another, whoever waits and however late.
+__device__ __forceinline__ void smem_count_release(uint32_t* c) {
+  asm volatile("red.release.cta.shared::cta.add.u32 [%0], 1;" ::"r"(smem_u32(c)) : "memory");
+}
+__device__ __forceinline__ uint32_t smem_count_acquire(const uint32_t* c) {
+  uint32_t v;
+  asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(c)) : "memory");
+  return v;
+}
+
 struct Smem {
   uint8_t* q;          // 2 buffers x (2 slabs x 128 rows x 128 B)
   uint8_t* k;          // STAGES x (2 slabs x 128 rows x 128 B)
@@ -247,6 +258,7 @@ struct Smem {
   uint64_t* lse_full;  // [2]
   uint64_t* lse_free;  // [2]
   uint32_t* tmem_holder;
+  uint32_t* a_cnt;     // statistics warps that have written their partial rows, over all pass-A ops
   float* lse;          // [2][128] denominators of the pairs of the current / next pass-B op
   ScoreOp* ops;        // [kSmemOps] the first ops of this CTA's program
 };
@@ -269,7 +281,8 @@ __device__ __forceinline__ Smem carve(uint8_t* base) {
   s.q_empty = (uint64_t*)p;   p += 16;
   s.lse_full = (uint64_t*)p;  p += 16;
   s.lse_free = (uint64_t*)p;  p += 16;
-  s.tmem_holder = (uint32_t*)p; p += 16;
+  s.tmem_holder = (uint32_t*)p; p += 8;
+  s.a_cnt = (uint32_t*)p;     p += 8;
   p = (uint8_t*)(((uintptr_t)p + 15) & ~(uintptr_t)15);
   s.lse = (float*)p;          p += 2 * 128 * 4;
   s.ops = (ScoreOp*)p;
@@ -309,6 +322,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     for (int i = 0; i < NBUF; ++i) { mbar_init(&S.acc_full[i], 1); mbar_init(&S.acc_empty[i], 4); }
     for (int i = 0; i < 2; ++i) { mbar_init(&S.q_full[i], 1); mbar_init(&S.q_empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&S.lse_full[i], 1); mbar_init(&S.lse_free[i], NSTATW); }
+    *S.a_cnt = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // the program of this CTA: a global read per op would put an L2 round trip on every op
@@ -455,6 +469,22 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     // fixed order and publishes the row's base-2 log-sum-exp and entropy term.
     if (P.pair_done) {
       bool ok = true;
+      // Publishes, in program order, every pass-A op of this CTA whose twelve partial row sets
+      // are written: one fence, then the op's count goes to its pair.
+      int pub_oi = op_lo;
+      uint32_t pub = 0;
+      auto publish = [&]() -> bool {               // true once every pass-A op is published
+        while (pub_oi < op_hi) {
+          const ScoreOp o = get_op(pub_oi);
+          if (o.nkeys <= 0 || o.phase) { ++pub_oi; continue; }
+          if (smem_count_acquire(S.a_cnt) < (uint32_t)NSTATW * (pub + 1u)) return false;
+          __threadfence();
+          if (lane == 0) atomicAdd(&P.pair_cnt[o.req * P.Hkv + o.g], (uint32_t)NSTATW);
+          ++pub;
+          ++pub_oi;
+        }
+        return true;
+      };
       for (int pair = 0; pair < P.n_pairs && ok; ++pair) {
         const int s_lo = P.pair_aseg[pair] * NWG, s_hi = P.pair_aseg[pair + 1] * NWG;
         bool waited = false;
@@ -466,6 +496,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             const uint32_t want = (uint32_t)(s_hi - s_lo) * 4u * P.epoch;   // one per warp
             const long long t0 = clock64();
             while (ld_acquire(&P.pair_cnt[pair]) < want) {
+              publish();
               if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
               __nanosleep(100);
             }
@@ -503,6 +534,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             atomicAdd(&P.pair_done[pair], 1u);
           }
         }
+      }
+      // ops that finish after this warp's last merge
+      const long long t0 = clock64();
+      while (ok && !publish()) {
+        if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); break; }
+        __nanosleep(100);
       }
     }
   } else if (warp == WARP_LSE) {
@@ -719,11 +756,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
           }
         }
-        // deliver this warp's 32 partial rows of the segment; the release orders them before
-        // the count without stalling the warp
+        // Deliver this warp's 32 partial rows of the segment.  Making them visible to the other
+        // CTAs takes a fence of a few thousand cycles; the merger warp pays it once per op for all
+        // twelve warps, which only tell it, inside the CTA, that their rows are written.
         __stcg(&P.rowpart[((size_t)op.seg * NWG + wg) * 128 + lane_row], make_float4(m, z, zwin, w));
         __syncwarp();
-        if (lane == 0) red_release_add(&P.pair_cnt[pair], 1u);
+        if (lane == 0) smem_count_release(S.a_cnt);
       }
     }
   }
