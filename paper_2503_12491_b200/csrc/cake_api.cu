@@ -61,7 +61,7 @@ void free_ctx(cake_ctx* c) {
   cudaFree(c->d_req); cudaFree(c->d_units); cudaFree(c->d_H); cudaFree(c->d_V); cudaFree(c->d_P);
   cudaFree(c->d_budget[0]); cudaFree(c->d_budget[1]); cudaFree(c->d_status);
   cudaFree(c->d_raw[0]); cudaFree(c->d_raw[1]);
-  cudaFree(c->d_fresh); cudaFree(c->d_lists); cudaFree(c->d_prefix); cudaFree(c->d_lstate);
+  cudaFree(c->d_fresh[0]); cudaFree(c->d_fresh[1]); cudaFree(c->d_lists); cudaFree(c->d_prefix); cudaFree(c->d_lstate);
   cudaFree(c->d_hist); cudaFree(c->d_fill); cudaFree(c->d_arrivals); cudaFree(c->d_headsum);
   cudaFree(c->d_pos_packed); cudaFree(c->d_bitmap); cudaFree(c->d_lse2);
   cudaFree(c->d_rowpart); cudaFree(c->d_colpart[0]); cudaFree(c->d_colpart[1]);
@@ -76,8 +76,14 @@ void free_ctx(cake_ctx* c) {
   if (c->ev_side) cudaEventDestroy(c->ev_side);
   for (int i = 0; i < 2; ++i) {
     if (c->ev_score[i]) cudaEventDestroy(c->ev_score[i]);
-    if (c->ev_tail[i]) cudaEventDestroy(c->ev_tail[i]);
+    if (c->ev_pool[i]) cudaEventDestroy(c->ev_pool[i]);
   }
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
+  if (c->ev_pool_side) cudaEventDestroy(c->ev_pool_side);
+  for (int i = 0; i < 2; ++i) if (c->ev_evict[i]) cudaEventDestroy(c->ev_evict[i]);
+  if (c->pool_st) cudaStreamDestroy(c->pool_st);
+  if (c->side2) cudaStreamDestroy(c->side2);
   if (c->side) cudaStreamDestroy(c->side);
   if (c->prof.spans) {
     for (int i = 0; i < c->prof.cap; ++i) {
@@ -90,16 +96,19 @@ void free_ctx(cake_ctx* c) {
   delete c;
 }
 
-// Orders the side stream after everything enqueued so far on the caller's stream.
+// Orders the internal streams after everything enqueued so far on the caller's stream.
 cudaError_t side_after(cake_ctx* c, cudaStream_t st) {
   cudaError_t e = cudaEventRecord(c->ev_main, st);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_main, 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(c->pool_st, c->ev_main, 0);
   return e;
 }
-// Orders the caller's stream after everything enqueued so far on the side stream.
+// Orders the caller's stream after everything enqueued so far on the internal streams.
 cudaError_t main_after_side(cake_ctx* c, cudaStream_t st) {
   cudaError_t e = cudaEventRecord(c->ev_side, c->side);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_side, 0);
+  if (e == cudaSuccess) e = cudaEventRecord(c->ev_pool_side, c->pool_st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_pool_side, 0);
   return e;
 }
 
@@ -170,11 +179,18 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   ok = ok && cudaMallocHost((void**)&x->h_units, sizeof(ScoreUnit) * x->max_units) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&x->upload_done, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&x->side, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&x->side2, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&x->pool_st, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&x->ev_pool_side, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; i < 2; ++i)
+    ok = ok && cudaEventCreateWithFlags(&x->ev_evict[i], cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&x->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&x->ev_join, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&x->ev_main, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&x->ev_side, cudaEventDisableTiming) == cudaSuccess;
   for (int i = 0; i < 2; ++i) {
     ok = ok && cudaEventCreateWithFlags(&x->ev_score[i], cudaEventDisableTiming) == cudaSuccess;
-    ok = ok && cudaEventCreateWithFlags(&x->ev_tail[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&x->ev_pool[i], cudaEventDisableTiming) == cudaSuccess;
   }
   ok = ok && dev_alloc(&x->d_req, R) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_units, x->max_units) == cudaSuccess;
@@ -186,7 +202,8 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   ok = ok && dev_alloc(&x->d_status, 1) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_raw[0], (size_t)c.n_kv_heads * T) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_raw[1], (size_t)c.n_kv_heads * T) == cudaSuccess;
-  ok = ok && dev_alloc(&x->d_fresh, (size_t)c.n_kv_heads * T) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_fresh[0], (size_t)c.n_kv_heads * T) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_fresh[1], (size_t)c.n_kv_heads * T) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_lists, (size_t)x->list_elems) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_prefix, (size_t)x->max_lists * (kBins + 1)) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_lstate, (size_t)x->max_lists) == cudaSuccess;
@@ -337,7 +354,8 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
   ctx->alloc_of_buf[0] = ctx->alloc_of_buf[1] = -1;
   ctx->last_alloc = -1;
   CAKE_CUDA_TRY(cudaMemsetAsync(ctx->d_status, 0, sizeof(int32_t), st));
-  ctx->tail_recorded[0] = ctx->tail_recorded[1] = false;
+  ctx->pool_recorded[0] = ctx->pool_recorded[1] = false;
+  ctx->evict_recorded[0] = ctx->evict_recorded[1] = false;
   CAKE_CUDA_TRY(side_after(ctx, st));
   return CAKE_OK;
 }
@@ -350,18 +368,24 @@ int32_t cake_score_layer(cake_ctx* ctx, int32_t layer, const void* q_win, const 
   if (layer != ctx->n_ind || ctx->n_evicted != layer) return CAKE_ERR_STATE;
   cudaStream_t st = (cudaStream_t)stream;
   const int par = layer & 1;
-  // the buffers of this parity were last read by the cascade of layer - 2
-  if (ctx->tail_recorded[par]) CAKE_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev_tail[par], 0));
+  // the score kernel's outputs of this parity were last read by the pooling of layer - 2; the rest
+  // of that layer's cascade works on its own data and may still be running
+  if (ctx->pool_recorded[par]) CAKE_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev_pool[par], 0));
   int32_t rc = ctx->use_tc ? launch_score_tc(ctx, layer, q_win, k, lse, st)
                            : launch_score_simt(ctx, layer, q_win, k, lse, st);
   if (rc != CAKE_OK) return rc;
-  // everything after the score kernel runs on the side stream, beside the next layer's scoring
+  // Pooling and the preference run on their own stream beside the next layer's scoring and
+  // beside the budgets and eviction of the layer before; the pooled buffer of this parity was
+  // last read by the eviction of layer - 2.
   CAKE_CUDA_TRY(cudaEventRecord(ctx->ev_score[par], st));
-  CAKE_CUDA_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_score[par], 0));
-  const int sp = prof_begin(ctx, CAKE_PROF_FINALIZE, ctx->side);
-  rc = launch_pool(ctx, layer, true, true, ctx->side);
-  prof_end(ctx, sp, ctx->side);
+  CAKE_CUDA_TRY(cudaStreamWaitEvent(ctx->pool_st, ctx->ev_score[par], 0));
+  if (ctx->evict_recorded[par]) CAKE_CUDA_TRY(cudaStreamWaitEvent(ctx->pool_st, ctx->ev_evict[par], 0));
+  const int sp = prof_begin(ctx, CAKE_PROF_FINALIZE, ctx->pool_st);
+  rc = launch_pool(ctx, layer, true, true, ctx->pool_st);
+  prof_end(ctx, sp, ctx->pool_st);
   if (rc != CAKE_OK) return rc;
+  CAKE_CUDA_TRY(cudaEventRecord(ctx->ev_pool[par], ctx->pool_st));
+  ctx->pool_recorded[par] = true;
   ctx->n_ind = layer + 1;
   if (ctx->n_pref < layer + 1) ctx->n_pref = layer + 1;
   return CAKE_OK;
@@ -371,7 +395,9 @@ int32_t cake_allocate(cake_ctx* ctx, int32_t stage, void* stream) {
   if (!ctx || ctx->n_req < 0) return ctx ? CAKE_ERR_STATE : CAKE_ERR_ARG;
   if (stage < 0 || stage >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
   if (stage >= ctx->n_pref) return CAKE_ERR_STATE;
-  (void)stream;                      // ordered by the side stream
+  (void)stream;                      // ordered by the internal streams
+  // the newest layer's preference comes from the pooling stream
+  if (ctx->pool_recorded[stage & 1]) CAKE_CUDA_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_pool[stage & 1], 0));
   const int sp = prof_begin(ctx, CAKE_PROF_ALLOCATE, ctx->side);
   int32_t rc = launch_allocate(ctx, stage, ctx->side);
   prof_end(ctx, sp, ctx->side);
@@ -392,8 +418,8 @@ int32_t cake_evict(cake_ctx* ctx, int32_t stage, void* stream) {
   int32_t rc = launch_evict(ctx, stage, ctx->side);
   prof_end(ctx, sp, ctx->side);
   if (rc != CAKE_OK) return rc;
-  CAKE_CUDA_TRY(cudaEventRecord(ctx->ev_tail[stage & 1], ctx->side));
-  ctx->tail_recorded[stage & 1] = true;
+  CAKE_CUDA_TRY(cudaEventRecord(ctx->ev_evict[stage & 1], ctx->side));
+  ctx->evict_recorded[stage & 1] = true;
   ctx->n_evicted = stage + 1;
   return CAKE_OK;
 }
@@ -435,7 +461,7 @@ int32_t cake_get_indicators(cake_ctx* ctx, int32_t layer, float* out, void* stre
   if (ctx->n_req < 0 || layer != ctx->n_ind - 1) return CAKE_ERR_STATE;
   if (ctx->total_tokens == 0) return CAKE_OK;
   CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
-  CAKE_CUDA_TRY(cudaMemcpyAsync(out, ctx->d_fresh,
+  CAKE_CUDA_TRY(cudaMemcpyAsync(out, ctx->d_fresh[layer & 1],
                                 sizeof(float) * ctx->cfg.n_kv_heads * ctx->total_tokens,
                                 cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
   return CAKE_OK;
@@ -462,13 +488,14 @@ int32_t cake_set_indicators(cake_ctx* ctx, int32_t layer, const float* in, void*
   // the previous stage may still read the pooled buffer on the side stream
   CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
   if (ctx->total_tokens > 0)
-    CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_fresh, in,
+    CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_fresh[layer & 1], in,
                                   sizeof(float) * ctx->cfg.n_kv_heads * ctx->total_tokens,
                                   cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
   CAKE_CUDA_TRY(side_after(ctx, (cudaStream_t)stream));
   // bucket histogram of the supplied values (they are taken as already pooled)
   const int32_t rc = launch_pool(ctx, layer, false, false, ctx->side);
   if (rc != CAKE_OK) return rc;
+  ctx->pool_recorded[layer & 1] = false;             // same stream as the budgets: nothing to wait for
   ctx->n_ind = layer + 1;
   return CAKE_OK;
 }
@@ -537,6 +564,7 @@ int32_t cake_profile_enable(cake_ctx* ctx, int32_t on) {
 int32_t cake_profile_read(cake_ctx* ctx, double* ms_out, int64_t* spans_out, void* stream) {
   if (!ctx || !ms_out || !spans_out) return CAKE_ERR_ARG;
   CAKE_CUDA_TRY(cudaStreamSynchronize(ctx->side));
+  CAKE_CUDA_TRY(cudaStreamSynchronize(ctx->pool_st));
   CAKE_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
   for (int k = 0; k < CAKE_PROF_KINDS; ++k) { ms_out[k] = 0.0; spans_out[k] = 0; }
   Profiler& p = ctx->prof;

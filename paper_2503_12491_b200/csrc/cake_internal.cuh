@@ -93,10 +93,16 @@ struct cake_ctx {
   // The cascade of layer l (pooling, preference, budgets, eviction) runs on an internal side
   // stream while the caller's stream already scores layer l+1; events order the two.
   cudaStream_t side;
+  cudaStream_t side2;               // older layers' thresholds of a stage, beside the newest layer's scatter
+  cudaStream_t pool_st;             // pooling + preference of layer l+1, beside the budgets and eviction of layer l
   cudaEvent_t ev_main, ev_side;     // scratch events: caller's stream -> side, side -> caller's
+  cudaEvent_t ev_fork, ev_join;     // side -> side2 and back
+  cudaEvent_t ev_pool_side;         // scratch event: pooling stream -> caller's
+  cudaEvent_t ev_evict[2];          // eviction stage of that parity has finished (it reads d_fresh of that parity)
+  bool evict_recorded[2];
   cudaEvent_t ev_score[2];          // score kernel of a layer of that parity has finished
-  cudaEvent_t ev_tail[2];           // eviction stage of that parity has finished
-  bool tail_recorded[2];
+  cudaEvent_t ev_pool[2];           // pooling (the last reader of the score outputs) of that parity has finished
+  bool pool_recorded[2];
   int32_t rows;            // R = G * S_w
   int64_t sel_budget;      // B' = B_total - L * S_w
   // ---- batch state (host) ----
@@ -125,7 +131,7 @@ struct cake_ctx {
   int32_t* d_budget[2];    // [max_requests][L] selectable budgets, double-buffered by stage parity
   int32_t* d_status;       // sticky device status word
   float* d_raw[2];         // [H_kv][max_total_tokens] un-pooled indicator, by layer parity
-  float* d_fresh;          // [H_kv][max_total_tokens] pooled indicator of the newest layer
+  float* d_fresh[2];       // [H_kv][max_total_tokens] pooled indicator of the newest layer, by layer parity
   uint2* d_lists;          // per (req, layer, head): n entries (ordered indicator key, position)
   int64_t list_elems;
   int32_t* d_prefix;       // [max_lists][kBins+1] bucket offsets of every list

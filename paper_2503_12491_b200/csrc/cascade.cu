@@ -760,7 +760,7 @@ int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, bool finalize, c
   const dim3 grid((unsigned)(ctx->n_split + F.units), c.n_kv_heads, ctx->n_req);
   const int r = c.pool_kernel / 2;
 #define CAKE_POOL_LAUNCH(RR)                                                                     \
-  pool_hist<RR><<<grid, PH_THREADS, 0, st>>>(ctx->d_raw[layer & 1], ctx->d_fresh, ctx->d_req,    \
+  pool_hist<RR><<<grid, PH_THREADS, 0, st>>>(ctx->d_raw[layer & 1], ctx->d_fresh[layer & 1], ctx->d_req,    \
                                              ctx->d_hist, ctx->d_arrivals, ctx->d_prefix,        \
                                              ctx->n_split, layer, c.n_layers, c.n_kv_heads,      \
                                              ctx->total_tokens, c.pool_kernel, c.pool_mode,      \
@@ -791,7 +791,7 @@ int32_t launch_evict(cake_ctx* ctx, int32_t stage, cudaStream_t st) {
   const cake_config& c = ctx->cfg;
   if (ctx->n_req == 0) return CAKE_OK;
   EvictArgs A;
-  A.fresh = ctx->d_fresh;
+  A.fresh = ctx->d_fresh[stage & 1];
   A.lists = ctx->d_lists;
   A.prefix_all = ctx->d_prefix;
   A.states = ctx->d_lstate;
@@ -801,12 +801,18 @@ int32_t launch_evict(cake_ctx* ctx, int32_t stage, cudaStream_t st) {
   A.cur = ctx->d_budget[stage & 1];
   A.stage = stage; A.L = c.n_layers; A.Hkv = c.n_kv_heads;
   A.T = ctx->total_tokens;
+  // The older layers' lists and the newest layer's list share nothing: the two kernels run side
+  // by side, the thresholds on a second internal stream that forks from and joins `st`.
   if (stage > 0) {
-    thresholds_old<<<dim3(c.n_kv_heads, stage, ctx->n_req), EV_THREADS, 0, st>>>(A);
+    CAKE_CUDA_TRY(cudaEventRecord(ctx->ev_fork, st));
+    CAKE_CUDA_TRY(cudaStreamWaitEvent(ctx->side2, ctx->ev_fork, 0));
+    thresholds_old<<<dim3(c.n_kv_heads, stage, ctx->n_req), EV_THREADS, 0, ctx->side2>>>(A);
     count_launch();
+    CAKE_CUDA_TRY(cudaEventRecord(ctx->ev_join, ctx->side2));
   }
   scatter_new<<<dim3(ctx->n_split, c.n_kv_heads, ctx->n_req), SC_THREADS, 0, st>>>(A);
   count_launch();
+  if (stage > 0) CAKE_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev_join, 0));
   return cuda_status(cudaGetLastError());
 }
 
