@@ -878,7 +878,7 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
   const int64_t T = n_req > 0 ? ctx->h_req[n_req - 1].cu + ctx->h_req[n_req - 1].N : 0;
   int64_t tilesA_total = 0;
   for (int r = 0; r < n_req; ++r) tilesA_total += (int64_t)Hkv * ((ctx->h_req[r].N + TILE - 1) / TILE);
-  const int n_cta = (int)(tilesA_total < ctx->n_sm_score ? tilesA_total : ctx->n_sm_score);
+  int n_cta = (int)(tilesA_total < ctx->n_sm_score ? tilesA_total : ctx->n_sm_score);
   ctx->n_tc_ctas = n_cta;
   ctx->n_tc_ops_full = ctx->n_tc_ops_b = 0;
   ctx->n_tc_asegs = ctx->n_tc_bsegs = 0;
@@ -895,6 +895,25 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
     wave_begin.push_back(n_pairs);
   }
   const int n_waves = (int)wave_begin.size() - 1;
+  // Every wave ends when its slowest CTA does, i.e. after ceil(tiles / CTAs) tiles, and both
+  // passes walk it.  Among the CTA counts down to three quarters of the SMs on offer, take the
+  // smallest one that reaches the minimum of the summed quotients: the SMs left over shorten
+  // nothing here and go to the cascade kernels that run beside this one.
+  {
+    std::vector<int64_t> w(n_waves, 0);
+    for (int wv = 0; wv < n_waves; ++wv)
+      for (int p = wave_begin[wv]; p < wave_begin[wv + 1]; ++p) w[wv] += (ctx->h_req[p / Hkv].N + TILE - 1) / TILE;
+    int64_t best = -1;
+    int best_n = n_cta;
+    for (int n = n_cta; n >= 1 && n >= n_cta - n_cta / 4; --n) {
+      int64_t steps = 0;
+      for (int wv = 0; wv < n_waves; ++wv) steps += (w[wv] + n - 1) / n;
+      if (best < 0 || steps <= best) { best = steps; best_n = n; }
+      else break;
+    }
+    n_cta = best_n;
+    ctx->n_tc_ctas = n_cta;
+  }
   std::vector<std::vector<ScoreOp>> full(n_cta), bonly(n_cta), wa(n_cta), wb(n_cta);
   std::vector<std::vector<std::vector<ScoreOp>>> wbs;      // pass-B ops of every wave, per CTA
   int32_t aseg = 0, bseg = 0;
