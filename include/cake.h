@@ -20,9 +20,9 @@
  *     cake_profile_read and cake_destroy, which say so.
  *   - Stream order.  cake_score_layer runs on the caller's stream.  Everything
  *     that follows a layer's scoring (pooling, preference, cake_allocate,
- *     cake_evict) is enqueued on a stream the context owns, ordered after that
+ *     cake_evict) is enqueued on streams the context owns, ordered after that
  *     layer's score kernel by events, so that it runs beside the scoring of the
- *     next layer.  cake_compact, every cake_get_* / cake_set_* call, cake_begin
+ *     following layers.  cake_compact, every cake_get_* / cake_set_* call, cake_begin
  *     and cake_status first make the stream they are given wait for that
  *     internal work.  Hence: results are ordered into the caller's stream by
  *     the call that hands them out, not by cake_allocate / cake_evict
