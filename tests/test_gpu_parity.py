@@ -270,6 +270,56 @@ def test_one_full_size_layer_of_the_128k_workload():
     cake.destroy()
 
 
+def test_four_full_size_layers_through_the_pipelined_cascade():
+    """Four layers of the 128K workload, enqueued back to back as the benchmark does: while layer
+    l+1 is scored, layer l is pooled, allocated and evicted on the library's own streams.  The
+    preferences, the budgets and every retained set are checked against the oracle's cascade, and
+    a second batch in the same context must give the same bits."""
+    full = synth.workload(4)
+    L = 4
+    w = synth.scaled(full, n_layers=L, total_budget=full.total_budget // full.n_layers * L)
+    qs, ks, vs = harness.device_inputs(w)
+    cake = harness.cake_for(w)
+    k_out, v_out, off, pos = cake.run(qs, ks, vs, w.cu_seqlens)
+    assert cake.status() == 0
+    first = (pos.clone(), off.clone(), k_out.clone())
+    N = w.seq_lens[0]
+    n = N - w.window
+    ref = [O.score_layer(to_np(qs[l][0]), to_np(ks[l]), gamma=w.gamma, pool_kernel=w.pool_kernel,
+                         tau1=w.tau1, tau2=w.tau2) for l in range(L)]
+    H, V, P = (x.cpu().numpy() for x in cake.get_preferences())
+    for l in range(L):
+        assert_close(H[0, l], ref[l]["H"], f"H of layer {l}")
+        assert_close(V[0, l], ref[l]["V"], f"V of layer {l}")
+        assert_close(P[0, l], ref[l]["P"], f"P of layer {l}")
+    c = O.cascade([r["indicator"] for r in ref], [r["P"] for r in ref],
+                  total_budget=w.total_budget, window=w.window, seq_len=N)
+    budgets = cake.get_budgets().cpu().numpy()[0]
+    assert budgets.sum() == w.total_budget
+    assert np.abs(budgets - c.budgets).max() <= 2, (budgets, c.budgets)
+    pb = harness.split_blocks(w, pos, off)
+    kb = harness.split_blocks(w, k_out, off)
+    for l in range(L):
+        b = int(budgets[l]) - w.window
+        for g in range(w.n_kv_heads):
+            got = pb[0][l][g].cpu().numpy()
+            assert len(got) == budgets[l] and np.all(np.diff(got) > 0)
+            assert np.array_equal(got[b:], np.arange(n, N))
+            want = O.topk_keep(ref[l]["indicator"][g], b)
+            diff = np.setxor1d(got[:b], want)
+            if diff.size:
+                thr = np.sort(ref[l]["indicator"][g])[::-1][b - 1]
+                rel = np.abs(ref[l]["indicator"][g][diff] - thr) / thr
+                assert rel.max() <= 2 * RTOL, (l, g, diff.size, rel.max())
+        g = l % w.n_kv_heads                               # one head's rows per layer, bit for bit
+        src = ks[l][g, torch.from_numpy(pb[0][l][g].cpu().numpy()).long().cuda()]
+        assert torch.equal(kb[0][l][g], src)
+    k2, v2, off2, pos2 = cake.run(qs, ks, vs, w.cu_seqlens)
+    assert cake.status() == 0
+    assert torch.equal(off2, first[1]) and torch.equal(pos2, first[0]) and torch.equal(k2, first[2])
+    cake.destroy()
+
+
 # ---------------------------------------------------------------- edge cases
 def small_w(**kw):
     base = synth.scaled(synth.workload(1), n_layers=2, seq_lens=(100,), total_budget=2 * 30)
