@@ -60,6 +60,12 @@ extern "C" {
 #define CAKE_DTYPE_BF16 1
 #define CAKE_POOL_MAX   0
 #define CAKE_POOL_AVG   1
+/* What the eviction indicator combines (Section 4.3; the alternatives are the
+ * rows of the paper's indicator ablation, Table "indicator_abl"). */
+#define CAKE_IND_MEAN_PLUS_VAR  0   /* Mean + gamma * Var, Eq. 11 (default) */
+#define CAKE_IND_MEAN           1   /* Mean only                            */
+#define CAKE_IND_VAR            2   /* Var only                             */
+#define CAKE_IND_MEAN_TIMES_VAR 3   /* Mean * Var                           */
 
 #define CAKE_MAX_LAYERS 128
 
@@ -82,6 +88,8 @@ typedef struct cake_config {
                                window included; must be >= n_layers * window              */
   int32_t max_requests;     /* capacity: requests per batch                               */
   int64_t max_total_tokens; /* capacity: T = sum of prompt lengths per batch              */
+  int32_t indicator_mode;   /* CAKE_IND_*: which combination of the window mean and
+                               variance scores a key; gamma is used by mode 0 only        */
 } cake_config;
 
 /* Allocates a context (device state and scratch sized from the capacities) on

@@ -118,17 +118,32 @@ def layer_preference(a_obs: np.ndarray, tau1: float, tau2: float,
 # --------------------------------------------------------------------------
 # eviction indicator                                      (Section 4.3, Eq. 11)
 # --------------------------------------------------------------------------
+INDICATOR_KINDS = ("mean+var", "mean", "var", "mean*var")
+
+
 def indicator_raw(a_obs: np.ndarray, n_kv_heads: int, gamma: float,
-                  ddof: int = 0) -> np.ndarray:
+                  ddof: int = 0, kind: str = "mean+var") -> np.ndarray:
     """I[g,n] = Mean_i(Abar[g,:,n]) + gamma * Var_i(Abar[g,:,n]) for the
     non-window tokens, Abar = attention averaged over the group's query heads.
-    [H_q][S_w][n] -> [H_kv][n]                                        (Eq. 11)"""
+    [H_q][S_w][n] -> [H_kv][n]                                        (Eq. 11)
+    `kind` selects the other combinations of the paper's indicator ablation
+    (Section 5.3, Table "indicator_abl"): the mean alone, the variance alone,
+    their product."""
+    assert kind in INDICATOR_KINDS
     Hq, Sw, n = a_obs.shape
     G = Hq // n_kv_heads
     abar = a_obs.reshape(n_kv_heads, G, Sw, n).mean(axis=1)
     if n == 0:
         return np.zeros((n_kv_heads, 0), dtype=F64)
-    return abar.mean(axis=1) + F64(gamma) * abar.var(axis=1, ddof=ddof)
+    mean = abar.mean(axis=1)
+    var = abar.var(axis=1, ddof=ddof)
+    if kind == "mean":
+        return mean
+    if kind == "var":
+        return var
+    if kind == "mean*var":
+        return mean * var
+    return mean + F64(gamma) * var
 
 
 def pool1d(x: np.ndarray, kernel: int, mode: str = "max") -> np.ndarray:
@@ -150,12 +165,12 @@ def pool1d(x: np.ndarray, kernel: int, mode: str = "max") -> np.ndarray:
 
 def score_layer(q_win: np.ndarray, k: np.ndarray, *, gamma: float, pool_kernel: int,
                 tau1: float = 1.0, tau2: float = 1.0, ddof: int = 0,
-                pool_mode: str = "max") -> Dict[str, object]:
+                pool_mode: str = "max", indicator: str = "mean+var") -> Dict[str, object]:
     """Everything one layer contributes before the cascade: pooled indicator
     [H_kv][n] and (H_l, V_l, P_l).                    (Algorithm 1, lines 4-5)"""
     a_obs = observed_attention(q_win, k)
     H, V, P = layer_preference(a_obs, tau1, tau2, ddof)
-    raw = indicator_raw(a_obs, k.shape[0], gamma, ddof)
+    raw = indicator_raw(a_obs, k.shape[0], gamma, ddof, indicator)
     return {"indicator": pool1d(raw, pool_kernel, pool_mode), "indicator_raw": raw,
             "H": H, "V": V, "P": P}
 

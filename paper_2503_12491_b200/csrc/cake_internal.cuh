@@ -192,6 +192,15 @@ int32_t launch_compact(cake_ctx* ctx, int32_t lo, int32_t hi, const LayerPtrs& p
 int32_t launch_get_positions(cake_ctx* ctx, int32_t req, int32_t layer, int32_t* out,
                              int64_t capacity, cudaStream_t st);
 
+// The eviction indicator of one key from the mean and variance of its window attention
+// (Section 4.3, Eq. 11, and the combinations of the paper's indicator ablation).
+__device__ __forceinline__ float combine_indicator(int mode, float gamma, float mean, float var) {
+  return mode == CAKE_IND_MEAN_PLUS_VAR ? fmaf(gamma, var, mean)
+         : mode == CAKE_IND_MEAN        ? mean
+         : mode == CAKE_IND_VAR         ? var
+                                        : mean * var;
+}
+
 // Tracing spans (no-ops unless cake_profile_enable was called).
 int prof_begin(cake_ctx* ctx, int kind, cudaStream_t st);
 void prof_end(cake_ctx* ctx, int span, cudaStream_t st);

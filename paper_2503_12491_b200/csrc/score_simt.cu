@@ -223,7 +223,7 @@ score_colstats_simt(const T* __restrict__ q_win, const T* __restrict__ k,
                     const ReqInfo* __restrict__ reqs, const ScoreUnit* __restrict__ units,
                     const float* __restrict__ lse2, float* __restrict__ raw,
                     float* __restrict__ colpart, int Hq, int Hkv, int Sw, int d, int64_t T_tokens,
-                    float scale2, float gamma, int ddof) {
+                    float scale2, float gamma, int ddof, int ind_mode) {
   extern __shared__ __align__(16) float smem[];
   const int G = Hq / Hkv, rows = G * Sw, rows8 = (rows + 7) / 8 * 8;
   const SmemLayout L = carve(smem, rows8, d);
@@ -289,7 +289,7 @@ score_colstats_simt(const T* __restrict__ q_win, const T* __restrict__ k,
     if (valid && q4 == 0) {
       const float mean = a1 * inv_sw;
       const float var = fmaxf(a2 * inv_sw - mean * mean, 0.f) * bessel;
-      raw[(size_t)g * T_tokens + rq.cu + key0 + key_l] = fmaf(gamma, var, mean);
+      raw[(size_t)g * T_tokens + rq.cu + key0 + key_l] = combine_indicator(ind_mode, gamma, mean, var);
 #pragma unroll
       for (int h = 0; h < 8; ++h) {
         if (h < G) {
@@ -353,7 +353,7 @@ int32_t run(cake_ctx* ctx, int32_t layer, const void* q_win, const void* k, cons
   score_colstats_simt<T><<<grid, NT, smem, st>>>(
       (const T*)q_win, (const T*)k, ctx->d_req, ctx->d_units, ctx->d_lse2, ctx->d_raw[layer & 1],
       ctx->d_colpart[layer & 1], c.n_q_heads, c.n_kv_heads, c.window, c.head_dim, ctx->total_tokens, scale2,
-      c.gamma, c.var_ddof);
+      c.gamma, c.var_ddof, c.indicator_mode);
   count_launch();
   prof_end(ctx, sp, st);
   return cuda_status(cudaGetLastError());

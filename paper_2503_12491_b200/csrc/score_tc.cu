@@ -76,6 +76,7 @@ struct TcParams {
   int n_pairs;
   int Hkv, Hq, Sw, rows, d;
   float scale2, gamma, bessel;
+  int ind_mode;                 // CAKE_IND_*
 };
 
 // ------------------------------------------------------------------ PTX
@@ -229,10 +230,6 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
   uint32_t v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
-}
-
-__device__ __forceinline__ void red_release_add(uint32_t* p, uint32_t v) {
-  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 // A counter in shared memory that only grows: a wait for "at least v" cannot mistake one round
@@ -585,7 +582,6 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const ScoreOp op = get_op(oi);
       if (op.nkeys <= 0) continue;
       const int ntiles = (op.nkeys + TILE - 1) / TILE;
-      const int pair = op.req * P.Hkv + op.g;
       if (op.phase) {
         // ---------------- pass B: thread = key, columns = rows r' = i*G + h
         const int slot = kb & 1;
@@ -649,7 +645,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
             const float mean = a1 * inv_g * inv_sw;
             const float var = fmaxf(a2 * inv_g * inv_g * inv_sw - mean * mean, 0.f) * P.bessel;
-            P.raw[op.base + j] = fmaf(P.gamma, var, mean);
+            P.raw[op.base + j] = combine_indicator(P.ind_mode, P.gamma, mean, var);
           }
         }
         __syncwarp();
@@ -1029,6 +1025,7 @@ int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const v
   P.Hkv = c.n_kv_heads; P.Hq = c.n_q_heads; P.Sw = c.window; P.rows = ctx->rows; P.d = c.head_dim;
   P.scale2 = kLog2e / sqrtf((float)c.head_dim);
   P.gamma = c.gamma;
+  P.ind_mode = c.indicator_mode;
   P.bessel = c.var_ddof ? (float)c.window / (float)(c.window - 1) : 1.f;
 
   const int sp = prof_begin(ctx, CAKE_PROF_SCORE, st);

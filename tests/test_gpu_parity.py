@@ -229,6 +229,27 @@ def test_end_to_end_own_indicators_differ_only_near_threshold(case):
     cake.destroy()
 
 
+@pytest.mark.parametrize("mode,kind", [(1, "mean"), (2, "var"), (3, "mean*var")])
+@pytest.mark.parametrize("name", ["tiny-fp32", "gqa-bf16"])
+def test_indicator_modes_of_the_ablation(name, mode, kind):
+    """The other combinations of window mean and variance (Section 5.3, Table "indicator_abl"),
+    on the fp32 SIMT path and the bf16 tensor-core path."""
+    w = SMALL_CASES[name]()
+    qs, ks, vs = harness.device_inputs(w, layers=[0])
+    cake = harness.cake_for(w, indicator_mode=mode)
+    cake.begin(w.cu_seqlens)
+    cake.score_layer(0, qs[0], ks[0])
+    ind = cake.get_indicators(0).cpu().numpy()
+    cu = w.cu_seqlens
+    for r, N in enumerate(w.seq_lens):
+        n = N - w.window
+        ref = O.score_layer(to_np(qs[0][r]), to_np(ks[0][:, cu[r]:cu[r + 1]]), gamma=w.gamma,
+                            pool_kernel=w.pool_kernel, tau1=w.tau1, tau2=w.tau2, indicator=kind)
+        assert_close(ind[:, cu[r]:cu[r] + n], ref["indicator"], f"{kind} indicator, request {r}")
+    assert cake.status() == 0
+    cake.destroy()
+
+
 # ------------------------------------------------ full size, as the benchmark launches it
 def test_one_full_size_layer_of_the_128k_workload():
     """Layer 0 of the 128K Llama-3.1-8B-shaped workload at full length, in the launch

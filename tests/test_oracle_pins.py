@@ -188,6 +188,41 @@ def test_indicator_matches_brute_force_and_gamma_zero_is_mean():
     assert np.allclose(g0, mean_attn, rtol=1e-13)
 
 
+def test_indicator_kinds_of_the_ablation():
+    """Mean, Var and Mean*Var (Section 5.3, Table "indicator_abl") against a loop-only brute
+    force, the two-row closed form, and the uniform-attention closed form."""
+    rng = np.random.default_rng(15)
+    q, k = rand_case(rng, Hq=6, Hkv=2, Sw=4, N=13, d=3)
+    A = brute_attention(q, k, G=3)
+    obs = O.observed_attention(q, k)
+    mean_b = brute_indicator(A, 2, 3, 4, 9, 0.0)
+    var_b = brute_indicator(A, 2, 3, 4, 9, 1.0) - mean_b
+    assert np.allclose(O.indicator_raw(obs, 2, gamma=99.0, kind="mean"), mean_b, rtol=1e-12)
+    assert np.allclose(O.indicator_raw(obs, 2, gamma=99.0, kind="var"), var_b, rtol=1e-9, atol=1e-18)
+    assert np.allclose(O.indicator_raw(obs, 2, gamma=99.0, kind="mean*var"), mean_b * var_b,
+                       rtol=1e-9, atol=1e-20)
+    # S_w = 2, one head: mean = (a+b)/2, var = ((a-b)/2)^2
+    q2, k2 = rand_case(rng, Hq=1, Hkv=1, Sw=2, N=8)
+    o2 = O.observed_attention(q2, k2)
+    a, b = o2[0, 0], o2[0, 1]
+    assert np.allclose(O.indicator_raw(o2, 1, 0.0, kind="var")[0], ((a - b) / 2) ** 2, rtol=1e-12)
+    assert np.allclose(O.indicator_raw(o2, 1, 0.0, kind="mean*var")[0],
+                       (a + b) / 2 * ((a - b) / 2) ** 2, rtol=1e-12)
+    # uniform attention: every key has the same mean and variance of 1/c_i
+    n, Sw = 37, 6
+    qu, ku, c = uniform_case(n, Sw)
+    ou = O.observed_attention(qu, ku)
+    assert np.allclose(O.indicator_raw(ou, 1, 5.0, kind="mean"), np.mean(1.0 / c), rtol=1e-13)
+    assert np.allclose(O.indicator_raw(ou, 1, 5.0, kind="var"), np.var(1.0 / c), rtol=1e-12)
+    assert np.allclose(O.indicator_raw(ou, 1, 5.0, kind="mean*var"),
+                       np.mean(1.0 / c) * np.var(1.0 / c), rtol=1e-12)
+    # score_layer hands the kind through; the default is Eq. 11
+    full = O.score_layer(q, k, gamma=3.0, pool_kernel=1)
+    assert np.allclose(full["indicator"], mean_b + 3.0 * var_b, rtol=1e-9)
+    assert np.allclose(O.score_layer(q, k, gamma=3.0, pool_kernel=1, indicator="var")["indicator"],
+                       var_b, rtol=1e-9, atol=1e-18)
+
+
 def test_two_row_variance_is_population():
     # S_w = 2: Var(a, b) = ((a-b)/2)^2 with ddof 0
     rng = np.random.default_rng(6)
