@@ -486,7 +486,7 @@ int32_t cake_set_indicators(cake_ctx* ctx, int32_t layer, const float* in, void*
   if (ctx->n_req < 0) return CAKE_ERR_STATE;
   if (layer < 0 || layer >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
   if (layer != ctx->n_ind || ctx->n_evicted != layer) return CAKE_ERR_STATE;
-  // the previous stage may still read the pooled buffer on the side stream
+  // earlier stages may still be working on the internal streams
   CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
   if (ctx->total_tokens > 0)
     CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->d_fresh[layer & 1], in,

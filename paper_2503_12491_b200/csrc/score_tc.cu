@@ -18,17 +18,18 @@
 //     A(wave 0), A(wave 1), B(wave 0), A(wave 2), B(wave 1), ... , B(last wave)
 // so pass B re-reads a wave's K from L2 shortly after pass A brought it in, and DRAM
 // sees K once.  Pass B of a pair needs the pair's softmax denominators, i.e. every
-// CTA's pass-A partial rows.  The merge is spread over the grid by rows: one spare warp
-// of CTA r % grid waits until all partials of the pair are delivered, loads row r's
-// partials in a single round trip, merges them and counts the row as done.  The pass A
+// CTA's pass-A partial rows.  The merge is spread over the grid by rows: the merger warp
+// of CTA (pair * rows + r) % grid waits until all partials of the pair are delivered, loads
+// row r's partials in a single round trip, merges them and counts the row as done.  The pass A
 // of the next wave sits between a pair's pass A and its pass B, so pass B's wait on
 // that count is normally already satisfied.
 //
 // Warp roles in a CTA of 512 threads: warps 0..11 are "statistics" warps in three groups of
 // four (a group takes every third accumulator tile, a warp owns 32 of its TMEM lanes, works
 // alone and writes its own partial results), warp 12 issues TMA loads, warp 13 owns the
-// tensor-memory allocation and issues the MMAs, warp 14 merges rows, warp 15 stages the
-// denominators of the next pass-B op in shared memory.  Every wait
+// tensor-memory allocation and issues the MMAs (both as converged warps with an elected lane),
+// warp 14 publishes this CTA's finished pass-A ops to the grid and merges rows, warp 15 stages
+// the denominators of the next pass-B op in shared memory.  Every wait
 // (mbarrier or flag) is bounded; a timed-out wait raises CAKE_ERR_TIMEOUT and the CTA
 // drains and exits.
 #include "cake_internal.cuh"
