@@ -250,6 +250,33 @@ def test_indicator_modes_of_the_ablation(name, mode, kind):
     cake.destroy()
 
 
+@pytest.mark.parametrize("reserve", ["0", "40", "74"])
+def test_score_is_the_same_for_any_share_of_the_sms(monkeypatch, reserve):
+    """The score kernel's grid (and with it the plan: slices, segments, merge owners) follows
+    the number of SMs left to the cascade kernels; the results must not."""
+    monkeypatch.setenv("CAKE_RESERVED_SMS", reserve)
+    w = SMALL_CASES["ragged"]()
+    qs, ks, vs = harness.device_inputs(w)
+    ref = oracle_scores(w, qs, ks)
+    cake = harness.cake_for(w)
+    cake.begin(w.cu_seqlens)
+    cu = w.cu_seqlens
+    for l in range(w.n_layers):
+        cake.score_layer(l, qs[l], ks[l])
+        ind = cake.get_indicators(l).cpu().numpy()
+        for r, N in enumerate(w.seq_lens):
+            n = N - w.window
+            assert_close(ind[:, cu[r]:cu[r] + n], ref[l][r]["indicator"], f"layer {l} request {r}")
+        cake.allocate(l)
+        cake.evict(l)
+    H, V, P = (x.cpu().numpy() for x in cake.get_preferences())
+    for l in range(w.n_layers):
+        for r in range(len(w.seq_lens)):
+            assert_close(P[r, l], ref[l][r]["P"], f"P of layer {l} request {r}")
+    assert cake.status() == 0
+    cake.destroy()
+
+
 # ------------------------------------------------ full size, as the benchmark launches it
 def test_one_full_size_layer_of_the_128k_workload():
     """Layer 0 of the 128K Llama-3.1-8B-shaped workload at full length, in the launch
