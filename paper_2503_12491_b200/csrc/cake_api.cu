@@ -210,13 +210,13 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   ok = ok && dev_alloc(&x->d_lstate, (size_t)x->max_lists) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_hist, (size_t)R * c.n_kv_heads * kBins) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_fill, (size_t)R * c.n_kv_heads * kBins) == cudaSuccess;
-  ok = ok && dev_alloc(&x->d_arrivals, (size_t)R * c.n_kv_heads + R) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_arrivals, 2 * (size_t)R * c.n_kv_heads + R) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_headsum, (size_t)R * c.n_q_heads * 2) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_pos_packed, (size_t)x->pos_packed_cap) == cudaSuccess;
   if (x->bitmap_words > 0) ok = ok && dev_alloc(&x->d_bitmap, (size_t)x->bitmap_words) == cudaSuccess;
   ok = ok && cudaMemset(x->d_hist, 0, sizeof(uint32_t) * R * c.n_kv_heads * kBins) == cudaSuccess;
   ok = ok && cudaMemset(x->d_fill, 0, sizeof(uint32_t) * R * c.n_kv_heads * kBins) == cudaSuccess;
-  ok = ok && cudaMemset(x->d_arrivals, 0, sizeof(uint32_t) * (R * c.n_kv_heads + R)) == cudaSuccess;
+  ok = ok && cudaMemset(x->d_arrivals, 0, sizeof(uint32_t) * (2 * R * c.n_kv_heads + R)) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_lse2, (size_t)R * c.n_q_heads * c.window) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_rowpart, (size_t)x->max_units * c.n_kv_heads * x->rows) == cudaSuccess;
   {

@@ -139,7 +139,9 @@ struct cake_ctx {
   int64_t max_lists;
   uint32_t* d_hist;        // [max_pairs][kBins] bucket histogram of the arriving layer (zero at rest)
   uint32_t* d_fill;        // [max_pairs][kBins] scatter cursors (zero at rest)
-  uint32_t* d_arrivals;    // [max_pairs] chunk counters, then [max_requests] head counters (zero at rest)
+  uint32_t* d_arrivals;    // zero at rest: [max_pairs] split counters of the scatter, [max_requests] head
+                           // counters of the preference, [max_pairs] split counters of the pooling (the
+                           // pooling of layer l+1 runs beside the scatter of layer l: separate counters)
   double* d_headsum;       // [max_requests][H_q][2] per-head entropy / variance sums of the layer
   int32_t n_split;         // largest nsplit of the batch
   int32_t* d_pos_packed;   // [packed rows bound] positions in packed row order

@@ -761,7 +761,7 @@ int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, bool finalize, c
   const int r = c.pool_kernel / 2;
 #define CAKE_POOL_LAUNCH(RR)                                                                     \
   pool_hist<RR><<<grid, PH_THREADS, 0, st>>>(ctx->d_raw[layer & 1], ctx->d_fresh[layer & 1], ctx->d_req,    \
-                                             ctx->d_hist, ctx->d_arrivals, ctx->d_prefix,        \
+                                             ctx->d_hist, ctx->d_arrivals + ctx->max_pairs + c.max_requests, ctx->d_prefix, \
                                              ctx->n_split, layer, c.n_layers, c.n_kv_heads,      \
                                              ctx->total_tokens, c.pool_kernel, c.pool_mode,      \
                                              do_pool ? 1 : 0, F)

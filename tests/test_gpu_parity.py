@@ -322,7 +322,7 @@ def test_four_full_size_layers_through_the_pipelined_cascade():
     """Four layers of the 128K workload, enqueued back to back as the benchmark does: while layer
     l+1 is scored, layer l is pooled, allocated and evicted on the library's own streams.  The
     preferences, the budgets and every retained set are checked against the oracle's cascade, and
-    a second batch in the same context must give the same bits."""
+    further batches in the same context must give the same bits."""
     full = synth.workload(4)
     L = 4
     w = synth.scaled(full, n_layers=L, total_budget=full.total_budget // full.n_layers * L)
@@ -362,9 +362,10 @@ def test_four_full_size_layers_through_the_pipelined_cascade():
         g = l % w.n_kv_heads                               # one head's rows per layer, bit for bit
         src = ks[l][g, torch.from_numpy(pb[0][l][g].cpu().numpy()).long().cuda()]
         assert torch.equal(kb[0][l][g], src)
-    k2, v2, off2, pos2 = cake.run(qs, ks, vs, w.cu_seqlens)
-    assert cake.status() == 0
-    assert torch.equal(off2, first[1]) and torch.equal(pos2, first[0]) and torch.equal(k2, first[2])
+    for _ in range(6):                                     # the internal streams overlap differently each time
+        k2, v2, off2, pos2 = cake.run(qs, ks, vs, w.cu_seqlens)
+        assert cake.status() == 0
+        assert torch.equal(off2, first[1]) and torch.equal(pos2, first[0]) and torch.equal(k2, first[2])
     cake.destroy()
 
 
