@@ -212,6 +212,29 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// Two fp32 values in one 64-bit register and the packed fp32x2 arithmetic on them: one
+// instruction issue for two FMAs or adds.  The statistics loops are bound by issue slots, not by
+// the FMA pipe, so halving their FFMA/FADD count matters although the pipe rate is the same.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 v;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+  return v;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
 // 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
@@ -565,7 +588,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
       const float4 v = __ldcg(reinterpret_cast<const float4*>(P.lse2 + (size_t)pair * 128) + lane);
-      reinterpret_cast<float4*>(S.lse + slot * 128)[lane] = v;
+      // stored negated: the statistics warps add them
+      reinterpret_cast<float4*>(S.lse + slot * 128)[lane] = make_float4(-v.x, -v.y, -v.z, -v.w);
       __syncwarp();
       if (lane == 0) mbar_arrive(&S.lse_full[slot]);
       ++kb;
@@ -603,6 +627,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           float s1[G], s2[G], hk[G], a2 = 0.f;
 #pragma unroll
           for (int h = 0; h < G; ++h) { s1[h] = 0.f; s2[h] = 0.f; hk[h] = 0.f; }
+          f32x2 s1p[(G + 1) / 2], s2p[(G + 1) / 2], hkp[(G + 1) / 2];   // the same, two heads per register
+#pragma unroll
+          for (int hp = 0; hp < (G + 1) / 2; ++hp) { s1p[hp] = 0ull; s2p[hp] = 0ull; hkp[hp] = 0ull; }
           for (int c0 = 0; c0 < P.rows; c0 += 32) {
             uint32_t r[32];
             tmem_ld32_issue(taddr + c0, r);
@@ -612,26 +639,60 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
               __syncwarp();
               if (lane == 0) mbar_arrive(&S.acc_empty[b]);
             }
-            // 32 columns = 32/G window rows x G heads
+            // 32 columns = 32/G window rows x G heads; ls = minus the rows' log-sum-exps
             float ls[32];
 #pragma unroll
             for (int q4 = 0; q4 < 8; ++q4) {
               const float4 l4 = reinterpret_cast<const float4*>(lse_s + c0)[q4];
               ls[q4 * 4 + 0] = l4.x; ls[q4 * 4 + 1] = l4.y; ls[q4 * 4 + 2] = l4.z; ls[q4 * 4 + 3] = l4.w;
             }
+            if constexpr (G % 2 == 0) {
+              // two heads per instruction
+              const f32x2 sc2 = pack2(P.scale2, P.scale2);
 #pragma unroll
-            for (int ii = 0; ii < 32 / G; ++ii) {
-              float a = 0.f;
+              for (int ii = 0; ii < 32 / G; ++ii) {
+                f32x2 asum = 0ull;
 #pragma unroll
-              for (int h = 0; h < G; ++h) {
-                const float tt = fmaf(__uint_as_float(r[ii * G + h]), P.scale2, -ls[ii * G + h]);
-                const float p = ex2(tt);
-                s1[h] += p;
-                s2[h] = fmaf(p, p, s2[h]);
-                if (kEntropyB) hk[h] = fmaf(p, tt, hk[h]);
-                a += p;
+                for (int hp = 0; hp < G / 2; ++hp) {
+                  const int c = ii * G + 2 * hp;
+                  const f32x2 tt2 = fma2(pack2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), sc2,
+                                         pack2(ls[c], ls[c + 1]));
+                  float t0, t1;
+                  unpack2(tt2, t0, t1);
+                  const f32x2 p2 = pack2(ex2(t0), ex2(t1));
+                  s1p[hp] = add2(s1p[hp], p2);
+                  s2p[hp] = fma2(p2, p2, s2p[hp]);
+                  if (kEntropyB) hkp[hp] = fma2(p2, tt2, hkp[hp]);
+                  asum = hp == 0 ? p2 : add2(asum, p2);
+                }
+                float a0, a1;
+                unpack2(asum, a0, a1);
+                const float a = a0 + a1;
+                a2 = fmaf(a, a, a2);
               }
-              a2 = fmaf(a, a, a2);
+            } else {
+#pragma unroll
+              for (int ii = 0; ii < 32 / G; ++ii) {
+                float a = 0.f;
+#pragma unroll
+                for (int h = 0; h < G; ++h) {
+                  const float tt = fmaf(__uint_as_float(r[ii * G + h]), P.scale2, ls[ii * G + h]);
+                  const float p = ex2(tt);
+                  s1[h] += p;
+                  s2[h] = fmaf(p, p, s2[h]);
+                  if (kEntropyB) hk[h] = fmaf(p, tt, hk[h]);
+                  a += p;
+                }
+                a2 = fmaf(a, a, a2);
+              }
+            }
+          }
+          if constexpr (G % 2 == 0) {
+#pragma unroll
+            for (int hp = 0; hp < G / 2; ++hp) {
+              unpack2(s1p[hp], s1[2 * hp], s1[2 * hp + 1]);
+              unpack2(s2p[hp], s2[2 * hp], s2[2 * hp + 1]);
+              if (kEntropyB) unpack2(hkp[hp], hk[2 * hp], hk[2 * hp + 1]);
             }
           }
           const int j = op.key0 + it * TILE + lane_row;          // key index inside the request
@@ -710,16 +771,23 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 z *= f; zwin *= f;
                 m = mn;
               }
-              float zc[4] = {0.f, 0.f, 0.f, 0.f}, wc[4] = {0.f, 0.f, 0.f, 0.f};
+              // two keys per instruction: four partial sums in two packed accumulators
+              const f32x2 sc2 = pack2(P.scale2, P.scale2), nm2 = pack2(-m, -m);
+              f32x2 zc[2] = {0ull, 0ull}, wc[2] = {0ull, 0ull};
 #pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const float tt = fmaf(__uint_as_float(r[e]), P.scale2, -m);
-                const float ee = ex2(tt);
-                zc[e & 3] += ee;
-                wc[e & 3] = fmaf(ee, tt, wc[e & 3]);
+              for (int e = 0; e < 32; e += 2) {
+                const f32x2 tt2 = fma2(pack2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), sc2, nm2);
+                float t0, t1;
+                unpack2(tt2, t0, t1);
+                const f32x2 ee2 = pack2(ex2(t0), ex2(t1));
+                zc[(e >> 1) & 1] = add2(zc[(e >> 1) & 1], ee2);
+                wc[(e >> 1) & 1] = fma2(ee2, tt2, wc[(e >> 1) & 1]);
               }
-              z += (zc[0] + zc[1]) + (zc[2] + zc[3]);
-              w += (wc[0] + wc[1]) + (wc[2] + wc[3]);
+              float z0, z1, w0, w1;
+              unpack2(add2(zc[0], zc[1]), z0, z1);
+              unpack2(add2(wc[0], wc[1]), w0, w1);
+              z += z0 + z1;
+              w += w0 + w1;
             } else {
               float cm = -CUDART_INF_F;
 #pragma unroll
