@@ -445,3 +445,24 @@ def test_run_request_end_to_end_small():
     # more preferred layers get at least as many slots
     order = np.argsort(P)
     assert np.all(np.diff(c.budgets[order]) >= 0)
+
+
+def test_oracle_results_on_the_tiny_workload_are_unchanged():
+    """A change detector, not a pin: the stored values were written by tests/golden/make_golden.py
+    from this oracle.  A failure means the oracle's arithmetic moved; regenerate the file only
+    together with the passage of the paper that justifies the change."""
+    import importlib.util
+    import json
+    import os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "make_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    now = mod.compute()
+    with open(os.path.join(here, "tiny_cascade.json")) as f:
+        stored = json.load(f)
+    assert now["budgets"] == stored["budgets"]
+    assert now["positions"] == stored["positions"]
+    for key in ("H", "V", "P"):
+        assert np.allclose(now[key], stored[key], rtol=1e-12, atol=0.0), key
+
