@@ -29,7 +29,8 @@ def _rank(rank, world, port, out):
 def test_two_replicas_report_the_slowest_time_and_the_summed_tokens():
     world = 2
     port = 29500 + os.getpid() % 1000
-    with mp.Manager() as mgr:
+    # a spawned manager: forking a process that already runs torch's threads is unsafe
+    with mp.get_context("spawn").Manager() as mgr:
         out = mgr.dict()
         mp.spawn(_rank, args=(world, port, out), nprocs=world, join=True)
         res = dict(out)
