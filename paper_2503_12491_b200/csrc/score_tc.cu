@@ -891,9 +891,11 @@ cudaError_t launch_g(bool entropy_b, int n_cta, cudaStream_t st, const CUtensorM
 // Cuts the `tiles` tiles of one (request, head) pair, which start at flat tile index `flat`
 // of a wave of `W` tiles shared by `n_cta` CTAs (slot c owns flat tiles
 // [c*W/n_cta, (c+1)*W/n_cta)), into per-slot segments; slot c belongs to CTA (c+rot)%n_cta.
+// With `split`, a slot's segment of two or more tiles becomes two ops (pad = 1: first half,
+// pad = 2: second half) that the program builder may place apart.
 void cut_pair(std::vector<std::vector<ScoreOp>>& per_cta, int rot, int n_cta, int64_t W, int64_t flat,
               int tiles, int keys, int req, int g, int phase, int32_t& seg_counter, int64_t base,
-              int n_obs) {
+              int n_obs, bool split = false) {
   int t0 = 0;
   while (t0 < tiles) {
     const int64_t f = flat + t0;
@@ -902,14 +904,20 @@ void cut_pair(std::vector<std::vector<ScoreOp>>& per_cta, int rot, int n_cta, in
     while (c > 0 && (int64_t)c * W / n_cta > f) --c;
     const int64_t share_end = (int64_t)(c + 1) * W / n_cta;
     const int t1 = (int)((share_end - flat) < tiles ? (share_end - flat) : tiles);
-    ScoreOp op;
-    op.base = base; op.n = n_obs; op.pad = 0;
-    op.req = req; op.g = g; op.key0 = t0 * TILE;
-    const int kend = t1 * TILE < keys ? t1 * TILE : keys;
-    op.nkeys = kend - t0 * TILE;
-    op.phase = phase;
-    op.seg = seg_counter++;
-    per_cta[(c + rot) % n_cta].push_back(op);
+    const int parts = (split && t1 - t0 >= 2) ? 2 : 1;
+    const int tm = t0 + (t1 - t0 + 1) / 2;
+    for (int part = 0; part < parts; ++part) {
+      const int a = part == 0 ? t0 : tm, b = (parts == 2 && part == 0) ? tm : t1;
+      ScoreOp op;
+      op.base = base; op.n = n_obs;
+      op.pad = parts == 2 ? part + 1 : 0;
+      op.req = req; op.g = g; op.key0 = a * TILE;
+      const int kend = b * TILE < keys ? b * TILE : keys;
+      op.nkeys = kend - a * TILE;
+      op.phase = phase;
+      op.seg = seg_counter++;
+      per_cta[(c + rot) % n_cta].push_back(op);
+    }
     t0 = t1;
   }
 }
@@ -931,7 +939,7 @@ int64_t tc_max_segments(const cake_config& c, int n_sm) {
   const int64_t bytes = (int64_t)c.n_kv_heads * c.max_total_tokens * c.head_dim * 2;
   int64_t waves = 2 * (bytes / kWaveBytes) + 2;
   if (waves > pairs) waves = pairs;
-  return pairs + waves * n_sm;
+  return pairs + (waves + 2) * n_sm;          // + the two waves whose ops are halved
 }
 
 // Builds the per-CTA programs of the batch in ctx->h_req[0..n_req): `full` = both passes
@@ -979,17 +987,27 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
     n_cta = best_n;
     ctx->n_tc_ctas = n_cta;
   }
-  std::vector<std::vector<ScoreOp>> full(n_cta), bonly(n_cta), wa(n_cta), wb(n_cta);
-  std::vector<std::vector<std::vector<ScoreOp>>> wbs;      // pass-B ops of every wave, per CTA
+  // Program of a CTA, by waves:  A0 A1 B0 A2 B1 ... A(n-1) B(n-2) B(n-1).  Pass B of a wave waits
+  // for the wave's merged denominators, which trail the slowest CTA's pass A by some 7 us; in
+  // the steady state the pass A in between covers that.  At the two ends it does not, so there
+  // (when the waves are single pairs, and there are at least four) one op is halved and its halves
+  // placed apart: A2's first half goes before B0, and B(n-3)'s second half goes after A(n-1).
+  std::vector<std::vector<std::vector<ScoreOp>>> was(n_waves), wbs(n_waves);   // [wave][CTA]
+  std::vector<std::vector<ScoreOp>> full(n_cta), bonly(n_cta);
   int32_t aseg = 0, bseg = 0;
   int32_t* pair_aseg = ctx->h_tc_index;                    // [pairs+1]
   int32_t* pair_bseg = ctx->h_tc_index + (n_pairs + 1);    // [pairs+1]
+  const bool ends = kWaveDepth == 1 && n_waves >= 4;
+  auto single = [&](int wv) { return wave_begin[wv + 1] - wave_begin[wv] == 1; };
+  const int split_a = ends && single(2) ? 2 : -1;
+  const int split_b = ends && single(n_waves - 3) ? n_waves - 3 : -1;
   int rot = 0;
   for (int wv = 0; wv < n_waves; ++wv) {
     int64_t WA = 0;
     for (int p = wave_begin[wv]; p < wave_begin[wv + 1]; ++p)
       WA += (ctx->h_req[p / Hkv].N + TILE - 1) / TILE;
-    for (int cta = 0; cta < n_cta; ++cta) { wa[cta].clear(); wb[cta].clear(); }
+    was[wv].assign(n_cta, {});
+    wbs[wv].assign(n_cta, {});
     int64_t fa = 0;
     for (int p = wave_begin[wv]; p < wave_begin[wv + 1]; ++p) {
       const int r = p / Hkv, g = p % Hkv;
@@ -998,26 +1016,41 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
       pair_aseg[p] = aseg;
       pair_bseg[p] = bseg;
       const int64_t base = (int64_t)g * T + rq.cu;
-      cut_pair(wa, rot, n_cta, WA, fa, ta, rq.N, r, g, 0, aseg, base, rq.n);
+      cut_pair(was[wv], rot, n_cta, WA, fa, ta, rq.N, r, g, 0, aseg, base, rq.n, wv == split_a);
       // pass B walks the same flat tile positions, so a CTA re-reads the tiles it brought in
-      if (tb > 0) cut_pair(wb, rot, n_cta, WA, fa, tb, rq.n, r, g, 1, bseg, base, rq.n);
+      if (tb > 0) cut_pair(wbs[wv], rot, n_cta, WA, fa, tb, rq.n, r, g, 1, bseg, base, rq.n, wv == split_b);
       fa += ta;
     }
     // a wave's remainder tiles land on different CTAs each time (golden-ratio stride)
     rot = (rot + (int)(n_cta * 0.381966) + 1) % n_cta;
-    wbs.push_back(wb);
-    for (int cta = 0; cta < n_cta; ++cta) {
-      full[cta].insert(full[cta].end(), wa[cta].begin(), wa[cta].end());
-      if (wv >= kWaveDepth) {
-        const std::vector<ScoreOp>& due = wbs[wv - kWaveDepth][cta];
-        full[cta].insert(full[cta].end(), due.begin(), due.end());
-      }
-      bonly[cta].insert(bonly[cta].end(), wb[cta].begin(), wb[cta].end());
-    }
   }
-  for (int wv = n_waves > kWaveDepth ? n_waves - kWaveDepth : 0; wv < n_waves; ++wv)
-    for (int cta = 0; cta < n_cta; ++cta)
-      full[cta].insert(full[cta].end(), wbs[wv][cta].begin(), wbs[wv][cta].end());
+  // which = 0: every op, 1: first halves and unsplit ops, 2: second halves
+  auto put = [&](std::vector<ScoreOp>& dst, const std::vector<ScoreOp>& src, int which) {
+    for (const ScoreOp& op : src)
+      if (which == 0 || (which == 1 && op.pad != 2) || (which == 2 && op.pad == 2)) dst.push_back(op);
+  };
+  for (int cta = 0; cta < n_cta; ++cta) {
+    for (int wv = 0; wv < n_waves; ++wv) {
+      // pass A of this wave
+      if (wv == split_a) {
+        put(full[cta], was[wv][cta], 1);                       // A2 first half
+        put(full[cta], wbs[wv - 2][cta], 0);                   // B0 (held back one slot)
+        put(full[cta], was[wv][cta], 2);                       // A2 second half
+      } else {
+        put(full[cta], was[wv][cta], 0);
+      }
+      // pass B of the wave kWaveDepth behind
+      if (split_b >= 0 && wv == split_b + 2) put(full[cta], wbs[split_b][cta], 2);   // B(n-3) second half, after A(n-1)
+      const int bw = wv - kWaveDepth;
+      if (bw >= 0 && !(split_a >= 0 && bw == split_a - 2 && wv == split_a - 1)) {
+        if (bw == split_b) put(full[cta], wbs[bw][cta], 1);    // B(n-3) first half in its usual place
+        else put(full[cta], wbs[bw][cta], 0);
+      }
+      put(bonly[cta], wbs[wv][cta], 0);
+    }
+    for (int wv = n_waves > kWaveDepth ? n_waves - kWaveDepth : 0; wv < n_waves; ++wv)
+      put(full[cta], wbs[wv][cta], 0);
+  }
   pair_aseg[n_pairs] = aseg;
   pair_bseg[n_pairs] = bseg;
   if (aseg > ctx->max_tc_segs || bseg > ctx->max_tc_segs) return CAKE_ERR_CAPACITY;
