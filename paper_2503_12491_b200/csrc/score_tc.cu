@@ -37,6 +37,7 @@
 #include <cuda.h>
 #include <math_constants.h>
 
+#include <algorithm>
 #include <vector>
 
 namespace cake {
@@ -78,6 +79,7 @@ struct TcParams {
   int Hkv, Hq, Sw, rows, d;
   float scale2, gamma, bessel;
   int ind_mode;                 // CAKE_IND_*
+  int merge_ways;               // rows the merger warp merges side by side: 1, or 4 when pairs are short
 };
 
 // ------------------------------------------------------------------ PTX
@@ -506,6 +508,67 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         }
         return true;
       };
+      if (P.merge_ways == 4) {
+        // Short pairs (a ragged batch, MHA): a wave holds several pairs whose rows have few
+        // partials each, so four rows, of four consecutive pairs, are merged side by side by
+        // eight lanes each, and the wave's denominators are ready four times sooner.
+        const int sub = lane >> 3, l8 = lane & 7;
+        for (int p0 = 0; p0 < P.n_pairs && ok; p0 += 4) {
+          const int pair = p0 + sub;
+          const bool have = pair < P.n_pairs;
+          const int s_lo = have ? P.pair_aseg[pair] * NWG : 0, s_hi = have ? P.pair_aseg[pair + 1] * NWG : 0;
+          const int r0 = have ? (int)((blockIdx.x + gridDim.x - (unsigned)(((long long)pair * P.rows) % gridDim.x)) % gridDim.x)
+                              : P.rows;
+          bool waited = false;
+          for (int r = r0;; r += gridDim.x) {
+            const bool active = have && r < P.rows;
+            if (!__any_sync(0xffffffffu, active)) break;
+            if (!waited) {
+              const uint32_t want = (uint32_t)(s_hi - s_lo) * 4u * P.epoch;
+              const long long t0 = clock64();
+              for (;;) {
+                const bool ready = !active || ld_acquire(&P.pair_cnt[pair]) >= want;
+                if (__all_sync(0xffffffffu, ready)) break;
+                publish();
+                if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
+                __nanosleep(100);
+              }
+              if (!ok) break;
+              waited = true;
+            }
+            float4 acc = make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
+            if (active) {
+              for (int base = s_lo; base < s_hi; base += 8 * 8) {
+                float4 pv[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                  const int sg = base + u * 8 + l8;
+                  pv[u] = sg < s_hi ? __ldcg(&P.rowpart[(size_t)sg * 128 + r])
+                                    : make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) acc = merge_rows(acc, pv[u]);
+              }
+            }
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) {               // inside the eight lanes of a row
+              float4 other;
+              other.x = __shfl_xor_sync(0xffffffffu, acc.x, o);
+              other.y = __shfl_xor_sync(0xffffffffu, acc.y, o);
+              other.z = __shfl_xor_sync(0xffffffffu, acc.z, o);
+              other.w = __shfl_xor_sync(0xffffffffu, acc.w, o);
+              acc = (lane & o) ? merge_rows(other, acc) : merge_rows(acc, other);
+            }
+            if (active && l8 == 0) {
+              const float lz = log2f(acc.y);
+              __stcg(&P.lse2[(size_t)pair * 128 + r], acc.x + lz);
+              __stcg(&P.hrow[(size_t)pair * 128 + r], (acc.w - lz * (acc.y - acc.z)) / acc.y);
+              __threadfence();
+              atomicAdd(&P.pair_done[pair], 1u);
+            }
+          }
+        }
+      } else
       for (int pair = 0; pair < P.n_pairs && ok; ++pair) {
         const int s_lo = P.pair_aseg[pair] * NWG, s_hi = P.pair_aseg[pair + 1] * NWG;
         bool waited = false;
@@ -1075,6 +1138,12 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
   ctx->n_tc_ops_b = o - ctx->n_tc_ops_full;
   ctx->n_tc_asegs = aseg;
   ctx->n_tc_bsegs = bseg;
+  // four rows at a time when there are pairs to take them from and a row has few partials
+  {
+    int max_segs = 0;
+    for (int p = 0; p < n_pairs; ++p) max_segs = std::max(max_segs, pair_aseg[p + 1] - pair_aseg[p]);
+    ctx->tc_merge_ways = (n_pairs >= 4 && max_segs * NWG <= 128) ? 4 : 1;
+  }
   return CAKE_OK;
 }
 
@@ -1128,6 +1197,7 @@ int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const v
   P.scale2 = kLog2e / sqrtf((float)c.head_dim);
   P.gamma = c.gamma;
   P.ind_mode = c.indicator_mode;
+  P.merge_ways = ctx->tc_merge_ways;
   P.bessel = c.var_ddof ? (float)c.window / (float)(c.window - 1) : 1.f;
 
   const int sp = prof_begin(ctx, CAKE_PROF_SCORE, st);
