@@ -79,7 +79,7 @@ struct TcParams {
   int Hkv, Hq, Sw, rows, d;
   float scale2, gamma, bessel;
   int ind_mode;                 // CAKE_IND_*
-  int merge_ways;               // rows the merger warp merges side by side: 1, or 4 when pairs are short
+  int merge_ways;               // rows the merger warp merges side by side: 1, or 2 or 4 when pairs are short
 };
 
 // ------------------------------------------------------------------ PTX
@@ -508,12 +508,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         }
         return true;
       };
-      if (P.merge_ways == 4) {
+      if (P.merge_ways > 1) {
         // Short pairs (a ragged batch, MHA): a wave holds several pairs whose rows have few
-        // partials each, so four rows, of four consecutive pairs, are merged side by side by
-        // eight lanes each, and the wave's denominators are ready four times sooner.
-        const int sub = lane >> 3, l8 = lane & 7;
-        for (int p0 = 0; p0 < P.n_pairs && ok; p0 += 4) {
+        // partials each, so the rows of `ways` (2 or 4) consecutive pairs are merged side by side,
+        // by 32 / ways lanes each, and the wave's denominators are ready that much sooner.
+        const int ways = P.merge_ways, lpr = 32 / ways;         // lanes per row
+        const int sub = lane / lpr, l8 = lane % lpr;
+        for (int p0 = 0; p0 < P.n_pairs && ok; p0 += ways) {
           const int pair = p0 + sub;
           const bool have = pair < P.n_pairs;
           const int s_lo = have ? P.pair_aseg[pair] * NWG : 0, s_hi = have ? P.pair_aseg[pair + 1] * NWG : 0;
@@ -538,11 +539,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
             float4 acc = make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
             if (active) {
-              for (int base = s_lo; base < s_hi; base += 8 * 8) {
+              for (int base = s_lo; base < s_hi; base += 8 * lpr) {
                 float4 pv[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                  const int sg = base + u * 8 + l8;
+                  const int sg = base + u * lpr + l8;
                   pv[u] = sg < s_hi ? __ldcg(&P.rowpart[(size_t)sg * 128 + r])
                                     : make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
                 }
@@ -550,8 +551,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 for (int u = 0; u < 8; ++u) acc = merge_rows(acc, pv[u]);
               }
             }
-#pragma unroll
-            for (int o = 4; o > 0; o >>= 1) {               // inside the eight lanes of a row
+            for (int o = lpr >> 1; o > 0; o >>= 1) {           // inside the lanes of a row
               float4 other;
               other.x = __shfl_xor_sync(0xffffffffu, acc.x, o);
               other.y = __shfl_xor_sync(0xffffffffu, acc.y, o);
@@ -1138,11 +1138,12 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
   ctx->n_tc_ops_b = o - ctx->n_tc_ops_full;
   ctx->n_tc_asegs = aseg;
   ctx->n_tc_bsegs = bseg;
-  // four rows at a time when there are pairs to take them from and a row has few partials
+  // several rows at a time when there are pairs to take them from and a row has few partials
   {
     int max_segs = 0;
     for (int p = 0; p < n_pairs; ++p) max_segs = std::max(max_segs, pair_aseg[p + 1] - pair_aseg[p]);
-    ctx->tc_merge_ways = (n_pairs >= 4 && max_segs * NWG <= 128) ? 4 : 1;
+    const int partials = max_segs * NWG;
+    ctx->tc_merge_ways = n_pairs < 4 ? 1 : partials <= 128 ? 4 : partials <= 256 ? 2 : 1;
   }
   return CAKE_OK;
 }
