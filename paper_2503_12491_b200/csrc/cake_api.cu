@@ -284,6 +284,10 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
   const bool same = ctx->n_req == n_req && n_req > 0 &&
                     memcmp(ctx->h_cu, cu, sizeof(int64_t) * (n_req + 1)) == 0;
   if (!same && n_req > 0) {
+    // From here on the host tables are rebuilt in place: until that has succeeded the context
+    // describes no batch at all, so a failure cannot leave it half in the old batch and half in
+    // the new one (a later cake_begin then rebuilds everything, and other calls are refused).
+    ctx->n_req = -1;
     if (ctx->upload_pending) {                    // staging buffers still feed an earlier copy
       CAKE_CUDA_TRY(cudaEventSynchronize(ctx->upload_done));
       ctx->upload_pending = false;
@@ -505,6 +509,9 @@ int32_t cake_set_preferences(cake_ctx* ctx, int32_t n_set, const double* P, void
   if (!ctx || !P) return CAKE_ERR_ARG;
   if (ctx->n_req < 0) return CAKE_ERR_STATE;
   if (n_set < 1 || n_set > ctx->cfg.n_layers) return CAKE_ERR_ARG;
+  // A layer that has been evicted stored only the entries its budget could still reach; a new
+  // preference could make that budget grow again (Proposition 1 would no longer hold).
+  if (ctx->n_evicted > 0) return CAKE_ERR_STATE;
   if (ctx->n_req > 0) {
     CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
     CAKE_CUDA_TRY(cudaMemcpy2DAsync(ctx->d_P, sizeof(double) * ctx->cfg.n_layers, P,

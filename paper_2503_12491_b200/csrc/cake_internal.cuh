@@ -204,6 +204,15 @@ __device__ __forceinline__ float combine_indicator(int mode, float gamma, float 
                                         : mean * var;
 }
 
+// Function attributes (the dynamic shared-memory limit) belong to a device: a flag per device,
+// so that a context on a second GPU sets them there too.
+constexpr int kOnceDevices = 64;
+struct PerDeviceOnce {
+  bool done[kOnceDevices] = {};
+  bool need(int device) const { return device < 0 || device >= kOnceDevices || !done[device]; }
+  void mark(int device) { if (device >= 0 && device < kOnceDevices) done[device] = true; }
+};
+
 // Tracing spans (no-ops unless cake_profile_enable was called).
 int prof_begin(cake_ctx* ctx, int kind, cudaStream_t st);
 void prof_end(cake_ctx* ctx, int span, cudaStream_t st);

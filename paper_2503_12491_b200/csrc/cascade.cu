@@ -718,8 +718,9 @@ thresholds_old(const EvictArgs A) {
   const int g = blockIdx.x, layer = blockIdx.y, req = blockIdx.z;
   const ReqInfo rq = A.reqs[req];
   const size_t lid = ((size_t)req * A.L + layer) * A.Hkv + g;
-  const int b = min(A.cur[(size_t)req * A.L + layer], rq.n);
   const ListState old = A.states[lid];
+  // a list never grows again (Proposition 1): entries beyond its earlier budget were not stored
+  const int b = min(min(A.cur[(size_t)req * A.L + layer], rq.n), old.kept);
   if (old.kept == b) return;                                   // budget unchanged
   set_threshold(A.prefix_all + lid * (kBins + 1),
                 A.lists + rq.list_off + ((size_t)layer * A.Hkv + g) * rq.n, b, old.bucket,

@@ -61,7 +61,7 @@ sorted_positions(const uint2* __restrict__ lists, const int32_t* __restrict__ pr
     for (int i = threadIdx.x; i < end; i += POS_THREADS) {
       const uint2 e = list[i];
       const bool keep = i < start || e.x > st.thr_key || (e.x == st.thr_key && (int32_t)e.y <= st.pos_cut);
-      if (keep) atomicOr(&bits[e.y >> 5], 1u << (e.y & 31));
+      if (keep && e.y < (uint32_t)rq.n) atomicOr(&bits[e.y >> 5], 1u << (e.y & 31));
     }
   }
   __syncthreads();
@@ -164,11 +164,11 @@ int32_t run_sorted_positions(cake_ctx* ctx, int req0, int n_req, int lo, int hi,
   for (int r = req0; r < req0 + n_req; ++r) max_n = ctx->h_req[r].n > max_n ? ctx->h_req[r].n : max_n;
   int need_words = (max_n + 31) / 32;
   int smem_words = need_words < kBitmapSmemWords ? need_words : kBitmapSmemWords;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr;
+  if (attr.need(ctx->device)) {
     CAKE_CUDA_TRY(cudaFuncSetAttribute(sorted_positions, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kBitmapSmemWords * 4));
-    attr_done = true;
+    attr.mark(ctx->device);
   }
   const int64_t ctas = (int64_t)c.n_kv_heads * (hi - lo) * n_req;
   if (need_words > kBitmapSmemWords &&

@@ -325,14 +325,14 @@ int32_t run(cake_ctx* ctx, int32_t layer, const void* q_win, const void* k, cons
   const int rows = ctx->rows;
   const size_t smem = smem_bytes(rows, c.head_dim);
   const float scale2 = 1.4426950408889634f / sqrtf((float)c.head_dim);
-  static bool attr_done[2] = {false, false};
+  static PerDeviceOnce attr[2];
   const int ti = sizeof(T) == 4 ? 0 : 1;
-  if (!attr_done[ti]) {
+  if (attr[ti].need(ctx->device)) {
     CAKE_CUDA_TRY(cudaFuncSetAttribute(score_rowstats_simt<T>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     CAKE_CUDA_TRY(cudaFuncSetAttribute(score_colstats_simt<T>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    attr_done[ti] = true;
+    attr[ti].mark(ctx->device);
   }
   const dim3 grid(ctx->n_units, c.n_kv_heads);
   const int64_t n_lse = (int64_t)ctx->n_req * c.n_q_heads * c.window;

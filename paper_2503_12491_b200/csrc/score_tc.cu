@@ -48,6 +48,7 @@ constexpr int STAGES = 4;            // K tiles in flight
 constexpr int NBUF = 3;              // accumulator buffers: 3 x 128 of the 512 TMEM columns
 constexpr int TMEM_Q_COL = NBUF * 128;   // + 64 columns: the window queries as pass A's A operand
 constexpr int NWG = kScoreGroups;    // statistics warp groups
+static_assert(NWG == NBUF, "one accumulator buffer per statistics group");
 constexpr int STAT_THREADS = NWG * 128;
 constexpr int TC_THREADS = STAT_THREADS + 128;  // + TMA, MMA, row-merger and denominator warps
 constexpr int WARP_TMA = NWG * 4, WARP_MMA = NWG * 4 + 1, WARP_MERGE = NWG * 4 + 2,
@@ -56,7 +57,7 @@ constexpr int NSTATW = NWG * 4;      // statistics warps
 constexpr int SLAB_BYTES = TILE * 128;   // one 64-element slab of a 128-row tile
 constexpr long long kSpinLimit = 4000000000ll;   // cycles (~2 s) before a wait gives up
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLazyMax = 8.f;      // pass A rescales only when the row max grows by 2^8
+constexpr float kChunkSumMax = 65536.f;   // a pass-A chunk sum beyond this moves the row's reference
 constexpr int64_t kWaveBytes = 32ll << 20;
 constexpr int kWaveDepth = 1;         // pass B of a wave follows pass A of the wave this far ahead
 
@@ -661,15 +662,25 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     // ------------------------------------------------ statistics warps
     // Every warp works alone: it owns TMEM lanes 32*quad.. of the tiles its group takes, writes
     // its own partial results and never waits for another statistics warp.
-    const int wg = warp >> 2;                       // takes tiles t with t % NWG == wg
+    // Group wg takes the tiles t with t % NWG == wg; with as many buffers as groups that is
+    // always buffer wg, whose "ready" barrier the group then meets in consecutive phases.
+    const int wg = warp >> 2;
     const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
     const int lane_row = quad * 32 + lane;          // accumulator lane (row in pass A, key in pass B)
-    uint32_t t = 0, kb = 0;
+    const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(wg * 128);
+    uint64_t* const my_full = &S.acc_full[wg];
+    uint64_t* const my_empty = &S.acc_empty[wg];
+    const int b = wg;
+    (void)b;
+    uint32_t tmod = 0;                              // tiles of the ops so far, modulo NWG
+    uint32_t fpar = 0, kb = 0;                      // phase parity of my_full; pass-B ops so far
     bool ok = true;
     for (int oi = op_lo; oi < op_hi; ++oi) {
       const ScoreOp op = get_op(oi);
       if (op.nkeys <= 0) continue;
       const int ntiles = (op.nkeys + TILE - 1) / TILE;
+      const int it0 = (int)((wg + NWG - tmod) % NWG);            // the group's first tile of the op
+      tmod = (tmod + (uint32_t)ntiles) % NWG;
       if (op.phase) {
         // ---------------- pass B: thread = key, columns = rows r' = i*G + h
         const int slot = kb & 1;
@@ -680,13 +691,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 #pragma unroll
         for (int h = 0; h < G; ++h) { vacc[h] = 0.f; hs[h] = 0.f; }
         const float inv_sw = 1.f / (float)P.Sw, inv_g = 1.f / (float)G;
-        for (int it = 0; it < ntiles; ++it, ++t) {
-          if ((int)(t % NWG) != wg) continue;
-          const int b = t % NBUF;
-          if (ok) ok = mbar_wait(&S.acc_full[b], (t / NBUF) & 1, P.status);
+        for (int it = it0; it < ntiles; it += NWG) {
+          if (ok) ok = mbar_wait(my_full, fpar, P.status);
+          fpar ^= 1u;
           if (!ok) continue;
           tc_fence_after();
-          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * 128);
           float s1[G], s2[G], hk[G], a2 = 0.f;
 #pragma unroll
           for (int h = 0; h < G; ++h) { s1[h] = 0.f; s2[h] = 0.f; hk[h] = 0.f; }
@@ -700,7 +709,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             if (c0 + 32 >= P.rows) {
               tc_fence_before();
               __syncwarp();
-              if (lane == 0) mbar_arrive(&S.acc_empty[b]);
+              if (lane == 0) mbar_arrive(my_empty);
             }
             // 32 columns = 32/G window rows x G heads; ls = minus the rows' log-sum-exps
             float ls[32];
@@ -795,19 +804,17 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const int i_row = lane_row / G;
         const int last = op.n + i_row;                 // last key this row may attend to
         float m = -CUDART_INF_F, z = 0.f, zwin = 0.f, w = 0.f;
-        for (int it = 0; it < ntiles; ++it, ++t) {
-          if ((int)(t % NWG) != wg) continue;
-          const int b = t % NBUF;
-          if (ok) ok = mbar_wait(&S.acc_full[b], (t / NBUF) & 1, P.status);
+        for (int it = it0; it < ntiles; it += NWG) {
+          if (ok) ok = mbar_wait(my_full, fpar, P.status);
+          fpar ^= 1u;
           if (!ok) continue;
           tc_fence_after();
-          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * 128);
           const int key0 = op.key0 + it * TILE;
           const bool interior = key0 + TILE <= op.n && it * TILE + TILE <= op.nkeys;
           if (quad * 32 >= P.rows) {                   // these TMEM lanes hold padding rows
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&S.acc_empty[b]);
+            if (lane == 0) mbar_arrive(my_empty);
             continue;
           }
 #pragma unroll 1
@@ -818,39 +825,49 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             if (c0 + 32 >= TILE) {
               tc_fence_before();
               __syncwarp();
-              if (lane == 0) mbar_arrive(&S.acc_empty[b]);
+              if (lane == 0) mbar_arrive(my_empty);
             }
             if (interior) {
-              float c4[4] = {__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]),
-                             __uint_as_float(r[3])};
+              // Every key is visible and observed.  The exponentials are taken against the row's
+              // running reference m without looking for the chunk's maximum first; a chunk whose
+              // sum comes out beyond kChunkSumMax (or not finite: m still -inf) holds a logit far
+              // above m and is done once more after m has moved to the chunk's maximum.  That is
+              // rare after the first tiles, and any reference within reach of the fp32 exponent
+              // range gives the same sums.
+              const f32x2 sc2 = pack2(P.scale2, P.scale2);
+              float zs, ws;
+#pragma unroll 1
+              for (int pass = 0;; ++pass) {
+                // two keys per instruction: four partial sums in two packed accumulators
+                const f32x2 nm2 = pack2(-m, -m);
+                f32x2 zc[2] = {0ull, 0ull}, wc[2] = {0ull, 0ull};
 #pragma unroll
-              for (int e = 4; e < 32; ++e) c4[e & 3] = fmaxf(c4[e & 3], __uint_as_float(r[e]));
-              const float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3])) * P.scale2;
-              if (cm > m + kLazyMax) {                        // rare after the first tiles
-                const float mn = cm;
+                for (int e = 0; e < 32; e += 2) {
+                  const f32x2 tt2 = fma2(pack2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), sc2, nm2);
+                  float t0, t1;
+                  unpack2(tt2, t0, t1);
+                  const f32x2 ee2 = pack2(ex2(t0), ex2(t1));
+                  zc[(e >> 1) & 1] = add2(zc[(e >> 1) & 1], ee2);
+                  wc[(e >> 1) & 1] = fma2(ee2, tt2, wc[(e >> 1) & 1]);
+                }
+                float z0, z1, w0, w1;
+                unpack2(add2(zc[0], zc[1]), z0, z1);
+                unpack2(add2(wc[0], wc[1]), w0, w1);
+                zs = z0 + z1;
+                ws = w0 + w1;
+                if (zs <= kChunkSumMax || pass > 0) break;
+                float cm = __uint_as_float(r[0]);
+#pragma unroll
+                for (int e = 1; e < 32; ++e) cm = fmaxf(cm, __uint_as_float(r[e]));
+                const float mn = cm * P.scale2;
                 const float f = ex2(m - mn);                  // 0 while m = -inf
                 const float dm = (m == -CUDART_INF_F) ? 0.f : (m - mn);
                 w = f * fmaf(dm, z - zwin, w);
                 z *= f; zwin *= f;
                 m = mn;
               }
-              // two keys per instruction: four partial sums in two packed accumulators
-              const f32x2 sc2 = pack2(P.scale2, P.scale2), nm2 = pack2(-m, -m);
-              f32x2 zc[2] = {0ull, 0ull}, wc[2] = {0ull, 0ull};
-#pragma unroll
-              for (int e = 0; e < 32; e += 2) {
-                const f32x2 tt2 = fma2(pack2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), sc2, nm2);
-                float t0, t1;
-                unpack2(tt2, t0, t1);
-                const f32x2 ee2 = pack2(ex2(t0), ex2(t1));
-                zc[(e >> 1) & 1] = add2(zc[(e >> 1) & 1], ee2);
-                wc[(e >> 1) & 1] = fma2(ee2, tt2, wc[(e >> 1) & 1]);
-              }
-              float z0, z1, w0, w1;
-              unpack2(add2(zc[0], zc[1]), z0, z1);
-              unpack2(add2(wc[0], wc[1]), w0, w1);
-              z += z0 + z1;
-              w += w0 + w1;
+              z += zs;
+              w += ws;
             } else {
               float cm = -CUDART_INF_F;
 #pragma unroll
@@ -934,17 +951,17 @@ EncodeTiledFn encode_fn() {
 
 
 template <int G>
-cudaError_t launch_g(bool entropy_b, int n_cta, cudaStream_t st, const CUtensorMap& qmap,
+cudaError_t launch_g(int device, bool entropy_b, int n_cta, cudaStream_t st, const CUtensorMap& qmap,
                      const CUtensorMap& kmap, const TcParams& P) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr;
+  if (attr.need(device)) {
     cudaError_t e = cudaFuncSetAttribute(score_fused_kernel<G, false>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(score_fused_kernel<G, true>,
                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr.mark(device);
   }
   if (entropy_b) score_fused_kernel<G, true><<<n_cta, TC_THREADS, kSmemBytes, st>>>(qmap, kmap, P);
   else           score_fused_kernel<G, false><<<n_cta, TC_THREADS, kSmemBytes, st>>>(qmap, kmap, P);
@@ -1143,7 +1160,23 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
     int max_segs = 0;
     for (int p = 0; p < n_pairs; ++p) max_segs = std::max(max_segs, pair_aseg[p + 1] - pair_aseg[p]);
     const int partials = max_segs * NWG;
-    ctx->tc_merge_ways = n_pairs < 4 ? 1 : partials <= 128 ? 4 : partials <= 256 ? 2 : 1;
+    int ways = n_pairs < 4 ? 1 : partials <= 128 ? 4 : partials <= 256 ? 2 : 1;
+    // The merger handles `ways` consecutive pairs at once and waits for the pass A of all of them.
+    // A CTA's program only guarantees A(w+1) before B(w): a group that reached from wave w into
+    // wave w+2 would make B(w) wait for an A(w+2) that comes after it.  So every group must lie
+    // in at most two adjacent waves.
+    std::vector<int> wave_of(n_pairs, 0);
+    for (int wv = 0; wv < n_waves; ++wv)
+      for (int p = wave_begin[wv]; p < wave_begin[wv + 1]; ++p) wave_of[p] = wv;
+    auto span_ok = [&](int wy) {
+      for (int p0 = 0; p0 < n_pairs; p0 += wy) {
+        const int p1 = std::min(n_pairs, p0 + wy) - 1;
+        if (wave_of[p1] - wave_of[p0] > kWaveDepth) return false;
+      }
+      return true;
+    };
+    while (ways > 1 && !span_ok(ways)) ways >>= 1;
+    ctx->tc_merge_ways = ways;
   }
   return CAKE_OK;
 }
@@ -1221,10 +1254,10 @@ int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const v
   cudaError_t e;
   const bool eb = lse != nullptr;
   switch (G) {
-    case 1: e = launch_g<1>(eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
-    case 2: e = launch_g<2>(eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
-    case 4: e = launch_g<4>(eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
-    default: e = launch_g<8>(eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
+    case 1: e = launch_g<1>(ctx->device, eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
+    case 2: e = launch_g<2>(ctx->device, eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
+    case 4: e = launch_g<4>(ctx->device, eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
+    default: e = launch_g<8>(ctx->device, eb, ctx->n_tc_ctas, st, qmap, kmap, P); break;
   }
   count_launch();
   prof_end(ctx, sp, st);

@@ -1,13 +1,16 @@
 """A reduced case of the eviction path, sized for profiler captures.
 
-    python -m paper_2503_12491_b200.profile_case [--workload 4] [--layers 2] [--steps 1]
+    python -m paper_2503_12491_b200.profile_case [--workload 4] [--layers 2] [--steps 1] [--lse]
 
 Runs the first `--layers` layers of a benchmark workload (same shapes per layer,
 budget scaled with the layer count) through begin / score / allocate / evict /
 compact.  Every layer's K is still larger than the L2 cache at workloads 4 and 5,
 so DRAM counters stay meaningful, while only a few GB are held on the device and
-a capture that replays each kernel many times ends by itself.  Prints the time
-of the last step; that figure is for orientation only, never a benchmark value.
+a capture that replays each kernel many times ends by itself.  With --lse the
+window rows' log-sum-exps are computed beforehand (plain torch, as a fused attention
+forward would hand them over) and passed to cake_score_layer, so the score kernel runs
+its column pass only.  Prints the time of the last step; that figure is for orientation
+only, never a benchmark value.
 """
 from __future__ import annotations
 
@@ -19,12 +22,29 @@ import torch
 from . import harness, synth
 
 
+def window_lse(w, q, k) -> torch.Tensor:
+    """Natural-log sum-exp of every window row's scaled logits over its visible keys:
+    the input a caller passes as `lse` ([n_req][H_q][S_w] fp32)."""
+    cu = w.cu_seqlens
+    out = torch.empty(len(w.seq_lens), w.n_q_heads, w.window, dtype=torch.float32, device=q.device)
+    for r, N in enumerate(w.seq_lens):
+        i = torch.arange(w.window, device=q.device)[:, None]
+        j = torch.arange(N, device=q.device)[None, :]
+        for g in range(w.n_kv_heads):
+            qg = q[r][g * w.group:(g + 1) * w.group].float()
+            s = torch.einsum("hid,jd->hij", qg, k[g, cu[r]:cu[r + 1]].float()) / (w.head_dim ** 0.5)
+            s = s.masked_fill(j > (N - w.window) + i, float("-inf"))
+            out[r, g * w.group:(g + 1) * w.group] = torch.logsumexp(s, dim=-1)
+    return out
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", type=int, default=4)
     ap.add_argument("--layers", type=int, default=2)
     ap.add_argument("--steps", type=int, default=1)
     ap.add_argument("--warmup", type=int, default=1)
+    ap.add_argument("--lse", action="store_true", help="supply the window rows' log-sum-exps")
     args = ap.parse_args()
 
     full = synth.workload(args.workload)
@@ -32,6 +52,7 @@ def main() -> None:
     w = synth.scaled(full, n_layers=L, total_budget=full.total_budget // full.n_layers * L)
     torch.cuda.set_device(0)
     qs, ks, vs = harness.device_inputs(w)
+    lses = [window_lse(w, qs[l], ks[l]) for l in range(L)] if args.lse else None
     cake = harness.cake_for(w)
     cake.begin(w.cu_seqlens)
     rows = cake.packed_rows_bound()
@@ -43,7 +64,15 @@ def main() -> None:
     for it in range(args.warmup + args.steps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        cake.run(qs, ks, vs, w.cu_seqlens, **bufs)
+        if lses is None:
+            cake.run(qs, ks, vs, w.cu_seqlens, **bufs)
+        else:
+            cake.begin(w.cu_seqlens)
+            for l in range(L):
+                cake.score_layer(l, qs[l], ks[l], lse=lses[l])
+                cake.allocate(l)
+                cake.evict(l)
+            cake.compact(ks, vs, **bufs)
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1)

@@ -234,6 +234,44 @@ def test_two_row_variance_is_population():
     assert np.allclose(raw[0], (a + b) / 2 + 2.0 * ((a - b) / 2) ** 2, rtol=1e-12)
 
 
+def test_two_row_variance_unbiased_and_its_hand_through_to_the_preference():
+    # S_w = 2 with ddof 1: Var(a, b) = (a-b)^2 / 2, twice the population value (Eq. 5, Eq. 11)
+    rng = np.random.default_rng(16)
+    q, k = rand_case(rng, Hq=2, Hkv=1, Sw=2, N=9)
+    obs = O.observed_attention(q, k)
+    for h in range(2):
+        a, b = obs[h, 0], obs[h, 1]
+        assert np.allclose(O.shift(obs, ddof=1)[h], np.sum((a - b) ** 2 / 2), rtol=1e-12)
+    assert np.allclose(O.shift(obs, ddof=1), 2.0 * O.shift(obs, ddof=0), rtol=1e-12)
+    # layer_preference hands ddof through to V (and only to V), Eq. 6
+    H0, V0, P0 = O.layer_preference(obs, tau1=0.7, tau2=1.3, ddof=0)
+    H1, V1, P1 = O.layer_preference(obs, tau1=0.7, tau2=1.3, ddof=1)
+    assert H1 == H0
+    want_V1 = np.mean([np.sum((obs[h, 0] - obs[h, 1]) ** 2 / 2) for h in range(2)])
+    assert math.isclose(V1, want_V1, rel_tol=1e-12) and math.isclose(V1, 2.0 * V0, rel_tol=1e-12)
+    assert math.isclose(P1, H0 ** (1 / 0.7) * want_V1 ** (1 / 1.3), rel_tol=1e-12)
+    # and score_layer hands it to both the preference and the indicator
+    full = O.score_layer(q, k, gamma=3.0, pool_kernel=1, tau1=0.7, tau2=1.3, ddof=1)
+    abar = obs.mean(axis=0)
+    assert np.allclose(full["indicator"][0], (abar[0] + abar[1]) / 2 + 3.0 * (abar[0] - abar[1]) ** 2 / 2,
+                       rtol=1e-12)
+    assert math.isclose(full["V"], want_V1, rel_tol=1e-12) and math.isclose(full["P"], P1, rel_tol=1e-12)
+
+
+def test_unbiased_variance_against_a_loop_for_wider_windows():
+    rng = np.random.default_rng(17)
+    q, k = rand_case(rng, Hq=2, Hkv=2, Sw=5, N=12)
+    obs = O.observed_attention(q, k)
+    n = obs.shape[2]
+    for h in range(2):
+        tot = 0.0
+        for j in range(n):
+            col = [obs[h, i, j] for i in range(5)]
+            mu = sum(col) / 5
+            tot += sum((c - mu) ** 2 for c in col) / 4
+        assert math.isclose(O.shift(obs, ddof=1)[h], tot, rel_tol=1e-12)
+
+
 # -------------------------------------------------------------------- pooling
 def test_pool_known_values():
     x = np.array([[1.0, 5.0, 2.0, 0.0, 3.0]])
@@ -258,6 +296,27 @@ def test_pool_properties_and_brute_force():
                 assert got[g, j] == want
         assert np.all(got >= x)
         assert O.pool1d(x, kp, "max").shape == x.shape
+
+
+def test_avg_pool_brute_force_with_zero_padding_at_both_ends():
+    """Average pooling: zero padding, divisor = kernel at every position, ends included."""
+    rng = np.random.default_rng(8)
+    x = rng.random((2, 11)) - 0.3
+    for kp in (3, 5, 7, 9):
+        got = O.pool1d(x, kp, "avg")
+        r = kp // 2
+        for g in range(2):
+            for j in range(11):
+                want = sum(x[g][t] for t in range(j - r, j + r + 1) if 0 <= t < 11) / kp
+                assert math.isclose(got[g, j], want, rel_tol=1e-13, abs_tol=1e-15)
+        # a constant input keeps its value only where the whole kernel fits
+        c = O.pool1d(np.full((1, 11), 2.0), kp, "avg")[0]
+        assert np.allclose(c[r:11 - r], 2.0) and math.isclose(c[0], 2.0 * (r + 1) / kp)
+        assert math.isclose(c[-1], 2.0 * (r + 1) / kp)
+    # a kernel wider than the input
+    short = np.array([[1.0, 2.0, 4.0]])
+    assert np.allclose(O.pool1d(short, 7, "avg"), [[7 / 7, 7 / 7, 7 / 7]])
+    assert np.array_equal(O.pool1d(short, 7, "max"), [[4, 4, 4]])
 
 
 # ------------------------------------------------------------------ allocator
