@@ -210,6 +210,31 @@ int32_t cake_profile_read(cake_ctx* ctx, double* ms_out, int64_t* spans_out, voi
  * SIMT kernels, negative on error. */
 int32_t cake_uses_tensor_cores(const cake_ctx* ctx);
 
+/* Bound, in SM clock cycles, of every wait inside the kernels (a CTA waiting for another CTA's
+ * partial results, or for one of its own barriers).  A wait that runs out sets the sticky device
+ * status CAKE_ERR_TIMEOUT; the kernel then drains and returns, and the context stays usable (the
+ * results of that batch are not).  0 restores the default of 4e9 cycles (about two seconds).
+ *
+ * The score kernel's CTAs wait for one another, so all of them must be resident at once: it is
+ * launched with at most one CTA per SM of the device.  Score launches of two contexts must
+ * therefore not overlap on one device (two streams, or two host threads): each would hold SMs
+ * the other waits for, and both would end with CAKE_ERR_TIMEOUT after the wait limit instead of
+ * a result.  Serialise them with stream order or events. */
+int32_t cake_set_wait_limit(cake_ctx* ctx, int64_t cycles);
+/* Test hook for the bounded waits: adds `delta` to the launch count that the cross-CTA waits of
+ * the following cake_score_layer calls expect, until the next cake_begin.  With delta != 0 no
+ * count ever matches, so every such wait runs out after the wait limit (set a short one first)
+ * and the launch ends with the device status CAKE_ERR_TIMEOUT. */
+int32_t cake_debug_skew_sync(cake_ctx* ctx, int32_t delta);
+
+/* Launch plan of cake_score_layer for the current batch, for tests and diagnostics (the plan is
+ * built on the host in cake_begin; nothing here touches the device).  out8 is a HOST array of 8
+ * int32: [0] 1 if the tensor-core kernels are used, [1] CTAs of the score kernel, [2] waves (groups
+ * of (request, KV head) pairs whose keys pass A and pass B share through L2), [3] rows the merger
+ * warps combine side by side (1, 2 or 4), [4] pass-A segments, [5] pass-B segments, [6] ops in the
+ * CTAs' programs, [7] SMs left to the cascade kernels.  Entries [1]..[6] are 0 on the SIMT path. */
+int32_t cake_plan_info(const cake_ctx* ctx, int32_t* out8);
+
 /* ---- selection without any allocation ------------------------------------- */
 /* The paper has no counterpart for this entry point; it exists for callers that are not
  * allowed to allocate device memory when they call in: code running inside another

@@ -29,7 +29,7 @@ EXPORTS = [
     "cake_get_preferences", "cake_get_budgets", "cake_get_positions", "cake_set_indicators",
     "cake_set_preferences", "cake_status", "cake_strerror", "cake_launch_count",
     "cake_profile_enable", "cake_profile_read", "cake_uses_tensor_cores",
-    "cake_select_positions_static",
+    "cake_select_positions_static", "cake_plan_info", "cake_set_wait_limit", "cake_debug_skew_sync",
 ]
 PROF_KINDS = ["score", "finalize", "allocate", "evict", "compact"]
 
@@ -86,6 +86,9 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.cake_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64), vp]
     lib.cake_uses_tensor_cores.argtypes = [vp]
     lib.cake_select_positions_static.argtypes = [vp, i32, i32, i32, vp, vp]
+    lib.cake_plan_info.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.cake_set_wait_limit.argtypes = [vp, i64]
+    lib.cake_debug_skew_sync.argtypes = [vp, i32]
     lib.cake_strerror.argtypes = [i32]
     lib.cake_strerror.restype = ctypes.c_char_p
     lib.cake_launch_count.argtypes = []
@@ -265,6 +268,19 @@ class Cake:
         s = ctypes.c_int32(0)
         _check(self.lib.cake_status(self._h, ctypes.byref(s), _stream()), "cake_status")
         return int(s.value)
+
+    def set_wait_limit(self, cycles: int) -> None:
+        _check(self.lib.cake_set_wait_limit(self._h, cycles), "cake_set_wait_limit")
+
+    def debug_skew_sync(self, delta: int) -> None:
+        _check(self.lib.cake_debug_skew_sync(self._h, delta), "cake_debug_skew_sync")
+
+    def plan_info(self) -> dict:
+        out = (ctypes.c_int32 * 8)()
+        _check(self.lib.cake_plan_info(self._h, out), "cake_plan_info")
+        keys = ["tensor_cores", "ctas", "waves", "merge_ways", "a_segments", "b_segments", "ops",
+                "reserved_sms"]
+        return {k: int(out[i]) for i, k in enumerate(keys)}
 
     def uses_tensor_cores(self) -> bool:
         return int(self.lib.cake_uses_tensor_cores(self._h)) == 1

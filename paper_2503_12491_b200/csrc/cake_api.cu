@@ -355,6 +355,7 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
   }
   ctx->n_req = n_req;
   ctx->total_tokens = T;
+  ctx->debug_epoch_skew = 0;
   ctx->n_ind = ctx->n_pref = ctx->n_evicted = 0;
   ctx->alloc_of_buf[0] = ctx->alloc_of_buf[1] = -1;
   ctx->last_alloc = -1;
@@ -591,6 +592,34 @@ int32_t cake_profile_read(cake_ctx* ctx, double* ms_out, int64_t* spans_out, voi
 int32_t cake_uses_tensor_cores(const cake_ctx* ctx) {
   if (!ctx) return CAKE_ERR_ARG;
   return ctx->use_tc ? 1 : 0;
+}
+
+int32_t cake_set_wait_limit(cake_ctx* ctx, int64_t cycles) {
+  if (!ctx || cycles < 0) return CAKE_ERR_ARG;
+  ctx->wait_limit_cycles = cycles;
+  return CAKE_OK;
+}
+
+int32_t cake_debug_skew_sync(cake_ctx* ctx, int32_t delta) {
+  if (!ctx) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0) return CAKE_ERR_STATE;
+  ctx->debug_epoch_skew = delta;
+  return CAKE_OK;
+}
+
+int32_t cake_plan_info(const cake_ctx* ctx, int32_t* out8) {
+  if (!ctx || !out8) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0) return CAKE_ERR_STATE;
+  const bool tc = ctx->use_tc;
+  out8[0] = tc ? 1 : 0;
+  out8[1] = tc ? ctx->n_tc_ctas : 0;
+  out8[2] = tc ? ctx->n_tc_waves : 0;
+  out8[3] = tc && ctx->n_tc_ctas > 0 ? ctx->tc_merge_ways : 0;
+  out8[4] = tc ? ctx->n_tc_asegs : 0;
+  out8[5] = tc ? ctx->n_tc_bsegs : 0;
+  out8[6] = tc ? ctx->n_tc_ops_full : 0;
+  out8[7] = ctx->n_sm - ctx->n_sm_score;
+  return CAKE_OK;
 }
 
 const char* cake_strerror(int32_t code) {

@@ -155,6 +155,9 @@ struct cake_ctx {
   bool use_tc;
   bool hhead_from_rows;    // entropy came from pass A (d_hrow) rather than from pass B partials
   int32_t n_tc_ctas, max_tc_segs, max_pairs;
+  int32_t n_tc_waves;             // waves of the current plan
+  int64_t wait_limit_cycles;      // bound of every device-side wait (0 = the default, about 2 s)
+  int32_t debug_epoch_skew;       // test hook: added to the launch count the cross-CTA waits expect
   int32_t n_tc_asegs, n_tc_bsegs;          // pass-A / pass-B segments per layer
   int32_t n_tc_ops_full, n_tc_ops_b, max_tc_ops;
   uint32_t tc_epoch;              // both-pass launches since cake_begin

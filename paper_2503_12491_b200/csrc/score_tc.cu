@@ -49,13 +49,14 @@ constexpr int NBUF = 3;              // accumulator buffers: 3 x 128 of the 512 
 constexpr int TMEM_Q_COL = NBUF * 128;   // + 64 columns: the window queries as pass A's A operand
 constexpr int NWG = kScoreGroups;    // statistics warp groups
 static_assert(NWG == NBUF, "one accumulator buffer per statistics group");
+static_assert(NWG * 4 <= 16, "a_done holds one counter per statistics warp");
 constexpr int STAT_THREADS = NWG * 128;
 constexpr int TC_THREADS = STAT_THREADS + 128;  // + TMA, MMA, row-merger and denominator warps
 constexpr int WARP_TMA = NWG * 4, WARP_MMA = NWG * 4 + 1, WARP_MERGE = NWG * 4 + 2,
               WARP_LSE = NWG * 4 + 3;
 constexpr int NSTATW = NWG * 4;      // statistics warps
 constexpr int SLAB_BYTES = TILE * 128;   // one 64-element slab of a 128-row tile
-constexpr long long kSpinLimit = 4000000000ll;   // cycles (~2 s) before a wait gives up
+constexpr long long kSpinLimit = 4000000000ll;   // default cycles (~2 s) before a wait gives up
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kChunkSumMax = 65536.f;   // a pass-A chunk sum beyond this moves the row's reference
 constexpr int64_t kWaveBytes = 32ll << 20;
@@ -76,6 +77,7 @@ struct TcParams {
   int32_t* status;
   int64_t T;
   uint32_t epoch;
+  long long spin_limit;         // cycles after which a wait gives up and raises CAKE_ERR_TIMEOUT
   int n_pairs;
   int Hkv, Hq, Sw, rows, d;
   float scale2, gamma, bessel;
@@ -111,11 +113,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false (and the sticky status set) if the phase never completes.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status,
+                                          long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kSpinLimit) {
+    if (clock64() - t0 > limit) {
       atomicCAS(status, 0, CAKE_ERR_TIMEOUT);
       return false;
     }
@@ -259,10 +262,10 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
   return v;
 }
 
-// A counter in shared memory that only grows: a wait for "at least v" cannot mistake one round
-// for another, whoever waits and however late.
-__device__ __forceinline__ void smem_count_release(uint32_t* c) {
-  asm volatile("red.release.cta.shared::cta.add.u32 [%0], 1;" ::"r"(smem_u32(c)) : "memory");
+// Counters in shared memory that only grow, each written by one warp: a wait for "at least v"
+// cannot mistake one round for another, whoever waits and however late.
+__device__ __forceinline__ void smem_store_release(uint32_t* c, uint32_t v) {
+  asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(c)), "r"(v) : "memory");
 }
 __device__ __forceinline__ uint32_t smem_count_acquire(const uint32_t* c) {
   uint32_t v;
@@ -282,14 +285,14 @@ struct Smem {
   uint64_t* lse_full;  // [2]
   uint64_t* lse_free;  // [2]
   uint32_t* tmem_holder;
-  uint32_t* a_cnt;     // statistics warps that have written their partial rows, over all pass-A ops
+  uint32_t* a_done;    // [NSTATW] pass-A ops whose partial rows each statistics warp has written
   float* lse;          // [2][128] denominators of the pairs of the current / next pass-B op
   ScoreOp* ops;        // [kSmemOps] the first ops of this CTA's program
 };
 
 constexpr size_t kQBytes = 2 * SLAB_BYTES;
 constexpr int kSmemOps = 128;        // ops of a CTA's program kept in shared memory
-constexpr size_t kSmemBytes = 1024 /*align*/ + 2 * kQBytes + (size_t)STAGES * 2 * SLAB_BYTES + 256 +
+constexpr size_t kSmemBytes = 1024 /*align*/ + 2 * kQBytes + (size_t)STAGES * 2 * SLAB_BYTES + 320 +
                               2 * 128 * 4 + kSmemOps * sizeof(ScoreOp) + 64;
 
 __device__ __forceinline__ Smem carve(uint8_t* base) {
@@ -306,7 +309,7 @@ __device__ __forceinline__ Smem carve(uint8_t* base) {
   s.lse_full = (uint64_t*)p;  p += 16;
   s.lse_free = (uint64_t*)p;  p += 16;
   s.tmem_holder = (uint32_t*)p; p += 8;
-  s.a_cnt = (uint32_t*)p;     p += 8;
+  s.a_done = (uint32_t*)p;    p += 4 * 16;
   p = (uint8_t*)(((uintptr_t)p + 15) & ~(uintptr_t)15);
   s.lse = (float*)p;          p += 2 * 128 * 4;
   s.ops = (ScoreOp*)p;
@@ -346,7 +349,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     for (int i = 0; i < NBUF; ++i) { mbar_init(&S.acc_full[i], 1); mbar_init(&S.acc_empty[i], 4); }
     for (int i = 0; i < 2; ++i) { mbar_init(&S.q_full[i], 1); mbar_init(&S.q_empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&S.lse_full[i], 1); mbar_init(&S.lse_free[i], NSTATW); }
-    *S.a_cnt = 0;
+    for (int i = 0; i < NSTATW; ++i) S.a_done[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // the program of this CTA: a global read per op would put an L2 round trip on every op
@@ -388,7 +391,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const uint64_t pol = (op.phase || !P.pair_done) ? drop : keep;
         const int qb = qn & 1;
         // the MMAs of the op that used this query buffer two ops ago must be done
-        ok = mbar_wait(&S.q_empty[qb], ((qn >> 1) & 1) ^ 1, P.status);
+        ok = mbar_wait(&S.q_empty[qb], ((qn >> 1) & 1) ^ 1, P.status, P.spin_limit);
         ++qn;
         if (!ok) break;
         mbar_expect_tx(&S.q_full[qb], (uint32_t)(P.rows * P.d * 2));
@@ -399,7 +402,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const int ntiles = (op.nkeys + TILE - 1) / TILE;
         for (int it = 0; it < ntiles; ++it, ++t) {
           const int s = t % STAGES;
-          ok = mbar_wait(&S.empty[s], ((t / STAGES) & 1) ^ 1, P.status);
+          ok = mbar_wait(&S.empty[s], ((t / STAGES) & 1) ^ 1, P.status, P.spin_limit);
           if (!ok) break;
           mbar_expect_tx(&S.full[s], stage_bytes);
           uint8_t* dst = S.k + (size_t)s * 2 * SLAB_BYTES;
@@ -411,9 +414,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       // do not leave the CTA while a bulk copy may still be writing its shared memory
       const uint32_t issued = t;
       for (uint32_t u = issued > STAGES ? issued - STAGES : 0; u < issued; ++u)
-        mbar_wait(&S.full[u % STAGES], (u / STAGES) & 1, P.status);
+        mbar_wait(&S.full[u % STAGES], (u / STAGES) & 1, P.status, P.spin_limit);
       for (uint32_t u = qn > 2 ? qn - 2 : 0; u < qn; ++u)
-        mbar_wait(&S.q_full[u & 1], (u >> 1) & 1, P.status);
+        mbar_wait(&S.q_full[u & 1], (u >> 1) & 1, P.status, P.spin_limit);
     }
   } else if (warp == WARP_MMA) {
     // ------------------------------------------------ MMA issuer (converged warp, elected lane issues)
@@ -426,7 +429,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         if (op.nkeys <= 0) continue;
         const uint32_t idesc = op.phase ? instr_desc(128, rows_pad) : instr_desc(128, TILE);
         const int qb = qn & 1;
-        ok = mbar_wait(&S.q_full[qb], (qn >> 1) & 1, P.status);
+        ok = mbar_wait(&S.q_full[qb], (qn >> 1) & 1, P.status, P.spin_limit);
         ++qn;
         if (!ok) break;
         const uint32_t qaddr = smem_u32(S.q + qb * kQBytes);
@@ -446,9 +449,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const int ntiles = (op.nkeys + TILE - 1) / TILE;
         for (int it = 0; it < ntiles; ++it, ++t) {
           const int s = t % STAGES, b = t % NBUF;
-          ok = mbar_wait(&S.acc_empty[b], ((t / NBUF) & 1) ^ 1, P.status);
+          ok = mbar_wait(&S.acc_empty[b], ((t / NBUF) & 1) ^ 1, P.status, P.spin_limit);
           if (!ok) break;
-          ok = mbar_wait(&S.full[s], (t / STAGES) & 1, P.status);
+          ok = mbar_wait(&S.full[s], (t / STAGES) & 1, P.status, P.spin_limit);
           if (!ok) break;
           tc_fence_after();
           const uint32_t k_lo = k_lo0 + (uint32_t)s * (uint32_t)((2 * SLAB_BYTES) >> 4);
@@ -501,7 +504,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         while (pub_oi < op_hi) {
           const ScoreOp o = get_op(pub_oi);
           if (o.nkeys <= 0 || o.phase) { ++pub_oi; continue; }
-          if (smem_count_acquire(S.a_cnt) < (uint32_t)NSTATW * (pub + 1u)) return false;
+          // every statistics warp counts its own finished pass-A ops: a warp whose group has
+          // no tile in an op runs ahead of the others, so a single shared count of arrivals
+          // could be reached before the slowest warp has written this op's rows
+          const uint32_t mine = lane < NSTATW ? smem_count_acquire(&S.a_done[lane]) : 0xFFFFFFFFu;
+          if (!__all_sync(0xffffffffu, mine >= pub + 1u)) return false;
           __threadfence();
           if (lane == 0) atomicAdd(&P.pair_cnt[o.req * P.Hkv + o.g], (uint32_t)NSTATW);
           ++pub;
@@ -532,7 +539,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 const bool ready = !active || ld_acquire(&P.pair_cnt[pair]) >= want;
                 if (__all_sync(0xffffffffu, ready)) break;
                 publish();
-                if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
+                if (clock64() - t0 > P.spin_limit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
                 __nanosleep(100);
               }
               if (!ok) break;
@@ -582,7 +589,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             const long long t0 = clock64();
             while (ld_acquire(&P.pair_cnt[pair]) < want) {
               publish();
-              if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
+              if (clock64() - t0 > P.spin_limit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
               __nanosleep(100);
             }
             if (!ok) break;
@@ -623,7 +630,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       // ops that finish after this warp's last merge
       const long long t0 = clock64();
       while (ok && !publish()) {
-        if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); break; }
+        if (clock64() - t0 > P.spin_limit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); break; }
         __nanosleep(100);
       }
     }
@@ -639,12 +646,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const int slot = kb & 1;
       const int pair = op.req * P.Hkv + op.g;
       if (lane == 0) {
-        ok = mbar_wait(&S.lse_free[slot], ((kb >> 1) & 1) ^ 1, P.status);
+        ok = mbar_wait(&S.lse_free[slot], ((kb >> 1) & 1) ^ 1, P.status, P.spin_limit);
         if (ok && P.pair_done) {
           const uint32_t want = (uint32_t)P.rows * P.epoch;
           const long long t0 = clock64();
           while (ld_acquire(&P.pair_done[pair]) < want) {
-            if (clock64() - t0 > kSpinLimit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
+            if (clock64() - t0 > P.spin_limit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
             __nanosleep(64);
           }
         }
@@ -674,6 +681,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     (void)b;
     uint32_t tmod = 0;                              // tiles of the ops so far, modulo NWG
     uint32_t fpar = 0, kb = 0;                      // phase parity of my_full; pass-B ops so far
+    uint32_t n_a_done = 0;                          // pass-A ops this warp has delivered
     bool ok = true;
     for (int oi = op_lo; oi < op_hi; ++oi) {
       const ScoreOp op = get_op(oi);
@@ -684,7 +692,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       if (op.phase) {
         // ---------------- pass B: thread = key, columns = rows r' = i*G + h
         const int slot = kb & 1;
-        if (ok) ok = mbar_wait(&S.lse_full[slot], (kb >> 1) & 1, P.status);
+        if (ok) ok = mbar_wait(&S.lse_full[slot], (kb >> 1) & 1, P.status, P.spin_limit);
         ++kb;
         const float* lse_s = S.lse + slot * 128;
         float vacc[G], hs[G];
@@ -692,7 +700,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         for (int h = 0; h < G; ++h) { vacc[h] = 0.f; hs[h] = 0.f; }
         const float inv_sw = 1.f / (float)P.Sw, inv_g = 1.f / (float)G;
         for (int it = it0; it < ntiles; it += NWG) {
-          if (ok) ok = mbar_wait(my_full, fpar, P.status);
+          if (ok) ok = mbar_wait(my_full, fpar, P.status, P.spin_limit);
           fpar ^= 1u;
           if (!ok) continue;
           tc_fence_after();
@@ -805,7 +813,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const int last = op.n + i_row;                 // last key this row may attend to
         float m = -CUDART_INF_F, z = 0.f, zwin = 0.f, w = 0.f;
         for (int it = it0; it < ntiles; it += NWG) {
-          if (ok) ok = mbar_wait(my_full, fpar, P.status);
+          if (ok) ok = mbar_wait(my_full, fpar, P.status, P.spin_limit);
           fpar ^= 1u;
           if (!ok) continue;
           tc_fence_after();
@@ -906,7 +914,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         // twelve warps, which only tell it, inside the CTA, that their rows are written.
         __stcg(&P.rowpart[((size_t)op.seg * NWG + wg) * 128 + lane_row], make_float4(m, z, zwin, w));
         __syncwarp();
-        if (lane == 0) smem_count_release(S.a_cnt);
+        ++n_a_done;
+        if (lane == 0) smem_store_release(&S.a_done[warp], n_a_done);
       }
     }
   }
@@ -1035,6 +1044,7 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
   ctx->n_tc_ctas = n_cta;
   ctx->n_tc_ops_full = ctx->n_tc_ops_b = 0;
   ctx->n_tc_asegs = ctx->n_tc_bsegs = 0;
+  ctx->n_tc_waves = 0;
   if (n_cta == 0) return CAKE_OK;
 
   std::vector<int> wave_begin{0};                          // waves of consecutive pairs
@@ -1048,6 +1058,7 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
     wave_begin.push_back(n_pairs);
   }
   const int n_waves = (int)wave_begin.size() - 1;
+  ctx->n_tc_waves = n_waves;
   // Every wave ends when its slowest CTA does, i.e. after ceil(tiles / CTAs) tiles, and both
   // passes walk it.  Among the CTA counts down to three quarters of the SMs on offer, take the
   // smallest one that reaches the minimum of the summed quotients: the SMs left over shorten
@@ -1232,6 +1243,7 @@ int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const v
   P.gamma = c.gamma;
   P.ind_mode = c.indicator_mode;
   P.merge_ways = ctx->tc_merge_ways;
+  P.spin_limit = ctx->wait_limit_cycles > 0 ? ctx->wait_limit_cycles : kSpinLimit;
   P.bessel = c.var_ddof ? (float)c.window / (float)(c.window - 1) : 1.f;
 
   const int sp = prof_begin(ctx, CAKE_PROF_SCORE, st);
@@ -1249,7 +1261,7 @@ int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const v
     ctx->hhead_from_rows = true;
     P.cta_op = cta_full;
     P.pair_done = ctx->d_tc_sync + ctx->max_pairs;
-    P.epoch = ++ctx->tc_epoch;
+    P.epoch = ++ctx->tc_epoch + (uint32_t)ctx->debug_epoch_skew;
   }
   cudaError_t e;
   const bool eb = lse != nullptr;
