@@ -26,20 +26,23 @@ if ROOT not in sys.path:
 METRIC = "CAKE score+evict+compact prompt tokens/s"
 # DRAM bytes of one score-kernel launch at workload 4 from the ncu capture under profiles/;
 # set to None whenever the kernel changes until the counters are taken again.
-SCORE_KERNEL_DRAM_BYTES = 282318080 + 10983936
+SCORE_KERNEL_DRAM_BYTES = None
 UNIT = "tokens/s"
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--blocks", type=int, default=10,
+                    help="timed blocks of --steps steps; the first one is the headline value, the "
+                         "others show the run-to-run spread")
     ap.add_argument("--workload", type=int, default=4, help="config index 1..5 (4 = 128K Llama-3.1-8B shape)")
     ap.add_argument("--impl", default="cake", choices=["cake", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-layers", type=int, default=1)
+    ap.add_argument("--cpu-sample-layers", type=int, default=2)
     return ap.parse_args()
 
 
@@ -68,7 +71,19 @@ class ClockSampler:
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
+
+    def median_between(self, t0: float, t1: float):
+        """Median sampled SM clock (MHz) of the samples taken in the host-time window."""
+        v = []
+        for ts, ln in list(self.lines):
+            if t0 <= ts <= t1:
+                try:
+                    v.append(float(ln.split(",")[0]))
+                except ValueError:
+                    pass
+        v.sort()
+        return v[len(v) // 2] if v else None
 
     def stop(self):
         if self.proc is None:
@@ -80,7 +95,7 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for _, ln in self.lines:
             p = [x.strip() for x in ln.split(",")]
             if len(p) < 6:
                 continue
@@ -97,67 +112,96 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------ CPU oracle leg
-def oracle_sample(w, sample_layers: int):
-    """Times the oracle, as it stands, on `sample_layers` full layers of the
-    workload's first request (score, budgets, top-k, compaction) and scales
-    to all layers.  Returns (tokens/s, seconds, threads, description)."""
-    import numpy as np
-    import torch
-    from oracle import cake_oracle as O
-    from paper_2503_12491_b200 import synth
-    try:
-        from threadpoolctl import threadpool_info
-        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
-    except Exception:
-        threads = os.cpu_count() or 1
-    N = w.seq_lens[0]
-    qs, ks, vs = [], [], []
-    w1 = synth.scaled(w, seq_lens=(N,))
-    for l in range(sample_layers):
-        q, k, v = synth.layer_inputs(w1, l, "cpu")
-        qs.append(q[0].float().numpy().astype(np.float64))
-        ks.append(k.float().numpy().astype(np.float64))
-        vs.append(v.float().numpy().astype(np.float64))
-    t0 = time.perf_counter()
-    scored = [O.score_layer(q, k, gamma=w.gamma, pool_kernel=w.pool_kernel, tau1=w.tau1, tau2=w.tau2)
-              for q, k in zip(qs, ks)]
-    # the sampled layers stand for all L: they share the budget the full cascade would give them
-    share = w.total_budget * sample_layers // w.n_layers
-    c = O.cascade([s["indicator"] for s in scored], [s["P"] for s in scored],
-                  total_budget=share, window=w.window, seq_len=N)
-    for l in range(sample_layers):
-        O.compact(ks[l], vs[l], c.positions[l])
-    dt = time.perf_counter() - t0
-    full = dt * w.n_layers / sample_layers * (w.total_tokens / N)
-    desc = (f"{sample_layers} of {w.n_layers} layers of request 0 (N={N}), all steps, float64 NumPy; "
-            f"time scaled by L/{sample_layers}" + (f" and by total/N tokens" if w.total_tokens != N else ""))
-    return w.total_tokens / full, dt, threads, desc
+class OracleSample:
+    """The oracle, as it stands, on a bounded sample of the workload: `sample_layers` full
+    layers of the first request through every step of the path (score, budgets, top-k,
+    compaction).  Inputs are generated once; `run()` times one pass over them.  The oracle is
+    single-process NumPy: the only parallelism is the BLAS thread pool inside its matrix
+    products, whose size is reported as `cores`."""
+
+    def __init__(self, w, sample_layers: int):
+        import numpy as np
+        from paper_2503_12491_b200 import synth
+        try:
+            from threadpoolctl import threadpool_info
+            self.threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        except Exception:
+            self.threads = os.cpu_count() or 1
+        self.w = w
+        self.layers = max(1, min(sample_layers, w.n_layers))
+        self.N = w.seq_lens[0]
+        w1 = synth.scaled(w, seq_lens=(self.N,))
+        self.qs, self.ks, self.vs = [], [], []
+        for l in range(self.layers):
+            q, k, v = synth.layer_inputs(w1, l, "cpu")
+            self.qs.append(q[0].float().numpy().astype(np.float64))
+            self.ks.append(k.float().numpy().astype(np.float64))
+            self.vs.append(v.float().numpy().astype(np.float64))
+        # tokens the sample stands for, in the metric's unit: `layers` of the L layers of N prompt
+        # tokens are N * layers / L prompt tokens' worth of the whole path
+        self.tokens = self.N * self.layers / w.n_layers
+        self.desc = (f"{self.layers} of {w.n_layers} layers of request 0 (N={self.N}), every step of the "
+                     f"path, float64 NumPy (single process; BLAS threads are its only parallelism); "
+                     f"a pass counts as N*{self.layers}/{w.n_layers} prompt tokens")
+
+    def run(self) -> float:
+        """One timed pass; returns seconds."""
+        from oracle import cake_oracle as O
+        w = self.w
+        t0 = time.perf_counter()
+        scored = [O.score_layer(q, k, gamma=w.gamma, pool_kernel=w.pool_kernel, tau1=w.tau1, tau2=w.tau2)
+                  for q, k in zip(self.qs, self.ks)]
+        # the sampled layers stand for all L: they share the budget the full cascade would give them
+        share = w.total_budget * self.layers // w.n_layers
+        c = O.cascade([s["indicator"] for s in scored], [s["P"] for s in scored],
+                      total_budget=share, window=w.window, seq_len=self.N)
+        for l in range(self.layers):
+            O.compact(self.ks[l], self.vs[l], c.positions[l])
+        return time.perf_counter() - t0
 
 
 def run_reference(args, w):
+    """The reference arm: the oracle alone on the host cores.  A step is one pass over the
+    bounded sample; `ms_per_step` is its measured time and `value` the prompt tokens that the
+    sample stands for per second (the same number as scaling the time to all layers)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    vals = []
+    smp = OracleSample(w, args.cpu_sample_layers)
     for _ in range(max(1, args.warmup)):
-        oracle_sample(w, args.cpu_sample_layers)
-    desc = threads = None
-    t_all = 0.0
-    for _ in range(args.steps):
-        v, dt, threads, desc = oracle_sample(w, args.cpu_sample_layers)
-        vals.append(v); t_all += dt
-    value = sum(vals) / len(vals)
-    ms = w.total_tokens / value * 1e3
+        smp.run()
+    times = [smp.run() for _ in range(args.steps)]
+    dt = sum(times) / len(times)
+    value = smp.tokens / dt
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "steps": args.steps, "warmup": max(1, args.warmup), "ms_per_step": dt * 1e3,
+        "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(w),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": smp.threads, "kind": "oracle",
+                         "sample": smp.desc, "sample_seconds": dt,
+                         "seconds_min_max": [min(times), max(times)],
+                         "whole_workload_ms_extrapolated": w.total_tokens / value * 1e3},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def block_stats(ms, mhz, steps):
+    """Spread of the per-step time over the repeated blocks (this rank), and time x clock."""
+    srt = sorted(ms)
+    med = srt[len(srt) // 2]
+    known = [(m, c) for m, c in zip(ms, mhz) if c]
+    out = {"n_blocks": len(ms), "steps_per_block": steps, "ms_per_step_median": med,
+           "ms_per_step_min": srt[0], "ms_per_step_max": srt[-1],
+           "ms_per_step_each": [round(x, 4) for x in ms],
+           "sm_mhz_median_each": mhz}
+    if known:
+        prod = sorted(m * c for m, c in known)
+        out["ms_x_mhz_median"] = prod[len(prod) // 2]
+    return out
 
 
 def workload_config(w):
@@ -250,15 +294,27 @@ def main():
     if rank == 0:
         sampler.start()
     launches0 = binding.launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    ev0.record()
-    for _ in range(args.steps):
-        step(bufs)
-    ev1.record()
-    barrier()
-    ms_total = ev0.elapsed_time(ev1)
+    def timed_block():
+        """K steps bracketed by barrier + synchronize; (device ms, host window)."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        h0 = time.time()
+        e0.record()
+        for _ in range(args.steps):
+            step(bufs)
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1), (h0, time.time())
+
+    ms_total, win0 = timed_block()                 # the headline: exactly K steps
     launches = binding.launch_count() - launches0
+    # the same block again and again: how much one block moves from run to run, with the clock
+    # sampled during each
+    block_ms, block_mhz = [ms_total / args.steps], [sampler.median_between(*win0) if rank == 0 else None]
+    for _ in range(max(0, args.blocks - 1)):
+        ms_b, win = timed_block()
+        block_ms.append(ms_b / args.steps)
+        block_mhz.append(sampler.median_between(*win) if rank == 0 else None)
     # second pass of the same K steps with every stage bracketed by CUDA events on the
     # launching stream: gives the per-kernel durations (the brackets cost a little, so the
     # headline value comes from the first pass)
@@ -299,6 +355,7 @@ def main():
                                   "launch of the reduced case is a full-size launch)",
                 "bytes_per_launch": per_launch_bytes, "ms_per_launch": dom_ms,
                 "launches_timed": prof[dom]["spans"],
+                "blocks": block_stats(block_ms, block_mhz, args.steps),
                 "phase_ms_per_step": phase_ms, "ms_per_step_with_brackets": ms_profiled,
                 "whole_step": {"ideal_bytes": ideal, "GBps": step_gbps,
                                "frac_of_measured_peak": step_gbps / hbm_peak,
@@ -314,9 +371,10 @@ def main():
     if not args.no_e2e:
         line["e2e"] = e2e_leg(args, w, cake, qs, ks, vs, bufs, world, barrier)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, dt, threads, desc = oracle_sample(w, args.cpu_sample_layers)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                "sample": desc, "sample_seconds": dt}
+        smp = OracleSample(w, args.cpu_sample_layers)
+        dt = smp.run()
+        line["cpu_baseline"] = {"value": smp.tokens / dt, "unit": UNIT, "cores": smp.threads,
+                                "kind": "oracle", "sample": smp.desc, "sample_seconds": dt}
     if rank == 0:
         print(json.dumps(line), flush=True)
     cake.destroy()
