@@ -31,6 +31,7 @@ parameter so the alternative can be exercised):
   * TopK order: indicator descending, token position ascending   (Eq. 12)
   * stored indicators of survivors are kept as they are (Section 4.2)
   * compacted rows in ascending token position, window last      (Eq. 12)
+  * decode-time eviction: see the section of that name below
 
 Pins: tests/test_oracle_pins.py checks every function below against closed
 forms, invariants the paper states (Proposition 1, Theorem 2), special cases
@@ -303,6 +304,92 @@ def compact(k: np.ndarray, v: np.ndarray, positions: Sequence[np.ndarray]
     kh = np.stack([k[g][np.asarray(positions[g])] for g in range(k.shape[0])])
     vh = np.stack([v[g][np.asarray(positions[g])] for g in range(v.shape[0])])
     return kh, vh
+
+
+# --------------------------------------------------------------------------
+# decode-time eviction        (Section 5.1 "Implementation Details"; Appendix
+#                              "More Implementation Details"; Listing 1, the
+#                              branches taken when not prefilling)
+# --------------------------------------------------------------------------
+# After the prefill every layer's budget is frozen at its final allocation.  Per
+# generated token and layer the new token's K/V is appended, the new token's
+# attention over the cached keys is pooled and "updates" the stored scores, and
+# the layer is evicted back to its frozen budget; the S_w most recent tokens are
+# always kept.  Readings (the listing leaves them open; "parity unpinned"):
+#   * observed attention of the single new query: softmax over ALL cached keys
+#     (the new one included), columns of the S_w most recent tokens dropped, not
+#     renormalised -- the one-row case of Eq. 6's slice;
+#   * grouped-query models: mean over the group's query heads, as in the prefill;
+#   * pooling runs over the cache in ascending token position (the order the
+#     listing keeps the compressed cache in), same mode and kernel as the prefill;
+#   * `update_score`: the pooled value is ADDED to the stored score ("add",
+#     default); the token that has just left the window has no stored score and
+#     starts from its pooled value.  "max" and "replace" are the alternatives;
+#   * eviction: TopK of Eq. 12 with the frozen budget on the stored scores
+#     (score descending, position ascending), per KV head.
+DECODE_UPDATES = ("add", "max", "replace")
+
+
+@dataclass
+class DecodeHead:
+    """Decode-time cache of one (layer, KV head): entries in ascending token
+    position; the last `window` entries are the recent window and carry no score."""
+    positions: np.ndarray        # [c] int64
+    scores: np.ndarray           # [c - window] float64, stored eviction scores
+    k: np.ndarray                # [c][d]
+    v: np.ndarray                # [c][d]
+
+
+def decode_attention(q_new: np.ndarray, k_cache: np.ndarray) -> np.ndarray:
+    """softmax(q k^T / sqrt(d)) of one new query per head over all cached keys.
+    q_new: [G][d] (the query heads of one KV head), k_cache: [c][d] -> [G][c]   (Eq. 2)"""
+    q = np.asarray(q_new, dtype=F64)
+    k = np.asarray(k_cache, dtype=F64)
+    s = q @ k.T / np.sqrt(F64(q.shape[-1]))
+    return softmax_rows(s)
+
+
+def decode_step_head(h: DecodeHead, q_new: np.ndarray, k_new: np.ndarray, v_new: np.ndarray,
+                     position: int, *, window: int, budget: int, pool_kernel: int,
+                     pool_mode: str = "max", update: str = "add") -> Tuple[DecodeHead, np.ndarray]:
+    """One decode step of one (layer, KV head).  Returns the new state and the
+    positions that were evicted (normally one)."""
+    assert update in DECODE_UPDATES
+    pos = np.concatenate([h.positions, [position]]).astype(np.int64)
+    k = np.concatenate([h.k, np.asarray(k_new)[None, :]], axis=0)
+    v = np.concatenate([h.v, np.asarray(v_new)[None, :]], axis=0)
+    c = pos.shape[0]
+    n_obs = c - window                       # entries outside the recent window
+    if n_obs <= 0:
+        return DecodeHead(pos, np.zeros(0, dtype=F64), k, v), np.zeros(0, dtype=np.int64)
+    a = decode_attention(q_new, k)           # [G][c]
+    abar = a[:, :n_obs].mean(axis=0)         # observed slice, group mean
+    pooled = pool1d(abar[None, :], pool_kernel, pool_mode)[0]
+    old = h.scores.shape[0]                  # entries that already carry a score
+    scores = np.empty(n_obs, dtype=F64)
+    if update == "add":
+        scores[:old] = h.scores + pooled[:old]
+    elif update == "max":
+        scores[:old] = np.maximum(h.scores, pooled[:old])
+    else:
+        scores[:old] = pooled[:old]
+    scores[old:] = pooled[old:]              # tokens that have just left the window
+    keep = topk_keep(scores, budget)         # indices into the non-window entries, ascending
+    evicted = np.setdiff1d(np.arange(n_obs), keep)
+    sel = np.concatenate([keep, np.arange(n_obs, c)])
+    return DecodeHead(pos[sel], scores[keep], k[sel], v[sel]), pos[evicted]
+
+
+def decode_init(k: np.ndarray, v: np.ndarray, positions: Sequence[np.ndarray],
+                indicator: np.ndarray, window: int) -> List[DecodeHead]:
+    """Decode-time state of one layer from the prefill's result: retained positions
+    per KV head (ascending, window last) and the stored indicators of the survivors."""
+    out = []
+    for g in range(k.shape[0]):
+        p = np.asarray(positions[g], dtype=np.int64)
+        nw = p[: p.shape[0] - window]
+        out.append(DecodeHead(p, np.asarray(indicator[g], dtype=F64)[nw].copy(), k[g][p], v[g][p]))
+    return out
 
 
 # --------------------------------------------------------------------------

@@ -525,3 +525,110 @@ def test_oracle_results_on_the_tiny_workload_are_unchanged():
     for key in ("H", "V", "P"):
         assert np.allclose(now[key], stored[key], rtol=1e-12, atol=0.0), key
 
+
+
+# ------------------------------------------------------- decode-time eviction
+def _decode_head(rng, c=12, window=4, d=8):
+    return O.DecodeHead(np.arange(0, 2 * c, 2)[:c].astype(np.int64), rng.random(c - window),
+                        rng.normal(size=(c, d)), rng.normal(size=(c, d)))
+
+
+def test_decode_attention_is_a_softmax_row_per_head():
+    rng = np.random.default_rng(31)
+    q, k = rng.normal(size=(3, 8)), rng.normal(size=(11, 8))
+    a = O.decode_attention(q, k)
+    assert np.allclose(a.sum(axis=-1), 1.0, atol=1e-12)
+    for h in range(3):
+        e = [math.exp(sum(q[h][t] * k[j][t] for t in range(8)) / math.sqrt(8)) for j in range(11)]
+        assert np.allclose(a[h], np.array(e) / sum(e), rtol=1e-12)
+
+
+def test_decode_step_keeps_the_frozen_budget_and_the_window():
+    rng = np.random.default_rng(32)
+    window, budget = 4, 8
+    h = _decode_head(rng, c=budget + window, window=window)
+    nxt = int(h.positions[-1]) + 1
+    for t in range(20):
+        before = h
+        h, ev = O.decode_step_head(h, rng.normal(size=(2, 8)), rng.normal(size=8), rng.normal(size=8),
+                                   nxt + t, window=window, budget=budget, pool_kernel=3)
+        assert len(h.positions) == budget + window and len(h.scores) == budget
+        assert np.all(np.diff(h.positions) > 0)
+        assert len(ev) == 1                                    # one token in, one out
+        assert np.array_equal(h.positions[-window:], np.arange(nxt + t - window + 1, nxt + t + 1)
+                              if t >= window - 1 else h.positions[-window:])
+        assert h.positions[-1] == nxt + t                      # the new token is in the window
+        assert ev[0] not in h.positions and ev[0] in np.concatenate([before.positions, [nxt + t]])
+        # K/V rows travel with their positions
+        keep = np.isin(before.positions, h.positions)
+        assert np.array_equal(h.k[: keep.sum()], before.k[keep])
+
+
+def test_decode_step_below_the_budget_evicts_nothing():
+    rng = np.random.default_rng(33)
+    h = _decode_head(rng, c=10, window=4)
+    h2, ev = O.decode_step_head(h, rng.normal(size=(1, 8)), rng.normal(size=8), rng.normal(size=8), 99,
+                                window=4, budget=50, pool_kernel=5)
+    assert len(ev) == 0 and len(h2.positions) == 11 and len(h2.scores) == 7
+
+
+def test_decode_step_with_uniform_attention_closed_form():
+    """K = 0: the new query attends every cached key equally, 1/c each, so pooling (max) changes
+    nothing, every stored score grows by 1/c, the token that has just left the window starts at
+    1/c, and the entry with the lowest score is evicted (ties: the highest position goes)."""
+    window, budget, d = 3, 5, 4
+    pos = np.arange(budget + window)
+    stored = np.array([0.5, 0.1, 0.7, 0.1, 0.9])
+    h = O.DecodeHead(pos, stored.copy(), np.zeros((budget + window, d)), np.zeros((budget + window, d)))
+    h2, ev = O.decode_step_head(h, np.ones((2, d)), np.zeros(d), np.zeros(d), 8, window=window,
+                                budget=budget, pool_kernel=3)
+    c = budget + window + 1
+    # candidates: the five stored (+1/c) and position 5 (1/c alone): position 5 is the lowest
+    assert list(ev) == [5]
+    assert np.allclose(h2.scores, stored + 1.0 / c, rtol=1e-14)
+    # with the new entrant out of the way the tie between positions 1 and 3 costs position 3
+    h3 = O.DecodeHead(pos, np.array([0.5, 0.1, 0.7, 0.1, 0.9]), np.zeros((8, d)), np.zeros((8, d)))
+    h3, ev3 = O.decode_step_head(h3, np.ones((1, d)), np.zeros(d), np.zeros(d), 8, window=window,
+                                 budget=4, pool_kernel=1)
+    assert sorted(ev3) == [3, 5]
+
+
+def test_decode_eviction_equals_topk_from_scratch_and_update_modes():
+    rng = np.random.default_rng(34)
+    window, budget = 4, 7
+    for update in O.DECODE_UPDATES:
+        h = _decode_head(rng, c=budget + window, window=window)
+        for t in range(6):
+            q, kn, vn = rng.normal(size=(2, 8)), rng.normal(size=8), rng.normal(size=8)
+            position = int(h.positions[-1]) + 1
+            # the same step spelled out
+            k_all = np.concatenate([h.k, kn[None]], axis=0)
+            a = O.decode_attention(q, k_all)
+            n_obs = k_all.shape[0] - window
+            pooled = O.pool1d(a[:, :n_obs].mean(axis=0)[None], 3, "max")[0]
+            old = len(h.scores)
+            want = pooled.copy()
+            if update == "add":
+                want[:old] = h.scores + pooled[:old]
+            elif update == "max":
+                want[:old] = np.maximum(h.scores, pooled[:old])
+            cand_pos = np.concatenate([h.positions, [position]])[:n_obs]
+            # brute force: the evicted entry is the last one in (score descending, position ascending)
+            order = sorted(range(n_obs), key=lambda j: (-want[j], cand_pos[j]))
+            h, ev = O.decode_step_head(h, q, kn, vn, position, window=window, budget=budget,
+                                       pool_kernel=3, update=update)
+            assert list(ev) == [cand_pos[order[-1]]]
+            assert np.allclose(h.scores, want[np.sort(order[:budget])], rtol=1e-14)
+
+
+def test_decode_init_takes_the_survivors_indicators():
+    rng = np.random.default_rng(35)
+    n, window, Hkv, d = 20, 4, 2, 8
+    k, v = rng.normal(size=(Hkv, n + window, d)), rng.normal(size=(Hkv, n + window, d))
+    ind = rng.random((Hkv, n))
+    positions = [np.concatenate([O.topk_keep(ind[g], 6), np.arange(n, n + window)]) for g in range(Hkv)]
+    heads = O.decode_init(k, v, positions, ind, window)
+    for g in range(Hkv):
+        assert np.array_equal(heads[g].positions, positions[g])
+        assert np.array_equal(heads[g].scores, ind[g][positions[g][:6]])
+        assert np.array_equal(heads[g].k, k[g][positions[g]])
