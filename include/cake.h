@@ -67,6 +67,12 @@ extern "C" {
 #define CAKE_IND_VAR            2   /* Var only                             */
 #define CAKE_IND_MEAN_TIMES_VAR 3   /* Mean * Var                           */
 
+/* How cake_decode_step combines a new token's pooled attention with a stored score (the
+ * appendix listing calls it "update_score" without defining it). */
+#define CAKE_DECODE_ADD      0   /* stored + pooled (default reading)  */
+#define CAKE_DECODE_MAX      1   /* max(stored, pooled)                */
+#define CAKE_DECODE_REPLACE  2   /* pooled                             */
+
 #define CAKE_MAX_LAYERS 128
 
 typedef struct cake_ctx cake_ctx;
@@ -209,6 +215,47 @@ int32_t cake_profile_read(cake_ctx* ctx, double* ms_out, int64_t* spans_out, voi
  * (bf16, G*S_w a multiple of 32 up to 128, G in {1,2,4,8}), 0 if it runs the fp32
  * SIMT kernels, negative on error. */
 int32_t cake_uses_tensor_cores(const cake_ctx* ctx);
+
+/* ---- decode-time eviction ------------------------------------------------------------
+ * Section 5.1 ("tokens are evicted during both prefilling and decoding"), Appendix "More
+ * Implementation Details" (every layer's budget is frozen at the prefill's final allocation)
+ * and the decode branches of the appendix listing.  After the last cake_evict of a batch:
+ *
+ *   cake_decode_begin   builds the decode cache: block (r,l) = rows row_offsets[r*L+l] ..
+ *                       row_offsets[r*L+l+1]-1 of k_cache / v_cache, laid out [H_kv][cap][d] with
+ *                       cap = len + 1 slots per head (len = the layer's retained length, window
+ *                       included); slots 0..len-1 receive the retained rows in ascending token
+ *                       position, slot len is free.  The stored indicators of the survivors
+ *                       become their decode scores.  k_cache and v_cache: device, caller-owned,
+ *                       at least cake_decode_rows_bound() rows of d elements; row_offsets_out:
+ *                       device int64 [n_req*L+1] (may be NULL).  This call synchronises
+ *                       `stream` once (it reads the final budgets back to size its kernels).
+ *   cake_decode_step    one generated token, one layer: q_new [n_req][H_q][d], k_new and v_new
+ *                       [n_req][H_kv][d].  Per KV head the new K/V row goes into the free slot;
+ *                       the new query's attention over the head's cap cached keys (softmax over
+ *                       all of them, the S_w most recent columns dropped, mean over the group's
+ *                       query heads) is pooled along ascending token position with the
+ *                       context's pooling mode and kernel; the pooled value is added to the
+ *                       stored score of every token outside the recent window (a token that has
+ *                       just left the window starts from its pooled value; CAKE_DECODE_* selects
+ *                       other readings); then the entry that comes last in the order (score
+ *                       descending, position ascending) among those tokens is evicted and its
+ *                       slot becomes the free one, so the head is back at its frozen budget.
+ *                       Rows never move; layers may be stepped in any order, each once per token.
+ *   cake_decode_get_state  entries of one (request, layer) in ascending token position:
+ *                       positions_out int32 [H_kv][len], scores_out fp32 [H_kv][len] (0 for the
+ *                       window entries), slots_out int32 [H_kv][len] (slot of each entry inside
+ *                       its head's cap slots); any may be NULL.
+ * A head with more than 200 KB / (4 * (G + 1)) slots (10239 at G = 4) does not fit the step
+ * kernel's shared memory: cake_decode_begin then returns CAKE_ERR_CAPACITY. */
+int64_t cake_decode_rows_bound(const cake_ctx* ctx);
+int32_t cake_decode_begin(cake_ctx* ctx, const void* const* k_layers, const void* const* v_layers,
+                          void* k_cache, void* v_cache, int64_t* row_offsets_out, int32_t update_mode,
+                          void* stream);
+int32_t cake_decode_step(cake_ctx* ctx, int32_t layer, const void* q_new, const void* k_new,
+                         const void* v_new, void* k_cache, void* v_cache, void* stream);
+int32_t cake_decode_get_state(cake_ctx* ctx, int32_t req, int32_t layer, int32_t* positions_out,
+                              float* scores_out, int32_t* slots_out, void* stream);
 
 /* Bound, in SM clock cycles, of every wait inside the kernels (a CTA waiting for another CTA's
  * partial results, or for one of its own barriers).  A wait that runs out sets the sticky device

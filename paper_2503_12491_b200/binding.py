@@ -30,6 +30,7 @@ EXPORTS = [
     "cake_set_preferences", "cake_status", "cake_strerror", "cake_launch_count",
     "cake_profile_enable", "cake_profile_read", "cake_uses_tensor_cores",
     "cake_select_positions_static", "cake_plan_info", "cake_set_wait_limit", "cake_debug_skew_sync",
+    "cake_decode_rows_bound", "cake_decode_begin", "cake_decode_step", "cake_decode_get_state",
 ]
 PROF_KINDS = ["score", "finalize", "allocate", "evict", "compact"]
 
@@ -87,6 +88,11 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.cake_uses_tensor_cores.argtypes = [vp]
     lib.cake_select_positions_static.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.cake_plan_info.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.cake_decode_rows_bound.argtypes = [vp]
+    lib.cake_decode_rows_bound.restype = i64
+    lib.cake_decode_begin.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, vp, vp, i32, vp]
+    lib.cake_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.cake_decode_get_state.argtypes = [vp, i32, i32, vp, vp, vp, vp]
     lib.cake_set_wait_limit.argtypes = [vp, i64]
     lib.cake_debug_skew_sync.argtypes = [vp, i32]
     lib.cake_strerror.argtypes = [i32]
@@ -95,7 +101,8 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.cake_launch_count.restype = i64
     for name in EXPORTS:
         fn = getattr(lib, name)
-        if name not in ("cake_packed_rows_bound", "cake_strerror", "cake_launch_count"):
+        if name not in ("cake_packed_rows_bound", "cake_strerror", "cake_launch_count",
+                        "cake_decode_rows_bound"):
             fn.restype = i32
     _lib = lib
     return lib
@@ -268,6 +275,39 @@ class Cake:
         s = ctypes.c_int32(0)
         _check(self.lib.cake_status(self._h, ctypes.byref(s), _stream()), "cake_status")
         return int(s.value)
+
+    # -- decode-time eviction
+    def decode_begin(self, k_layers, v_layers, update_mode: int = 0):
+        """Builds the decode cache; returns (k_cache, v_cache, row_offsets)."""
+        L = self.cfg.n_layers
+        rows = int(self.lib.cake_decode_rows_bound(self._h))
+        if rows < 0:
+            raise CakeError(rows, "cake_decode_rows_bound")
+        dev = torch.device("cuda", torch.cuda.current_device())
+        k_cache = torch.zeros(max(rows, 1), self.cfg.head_dim, dtype=self.dtype, device=dev)
+        v_cache = torch.zeros(max(rows, 1), self.cfg.head_dim, dtype=self.dtype, device=dev)
+        off = torch.empty(self.n_req * L + 1, dtype=torch.int64, device=dev)
+        kp = (ctypes.c_void_p * L)(*[_ptr(t, self.dtype) for t in k_layers])
+        vp = (ctypes.c_void_p * L)(*[_ptr(t, self.dtype) for t in v_layers])
+        _check(self.lib.cake_decode_begin(self._h, kp, vp, _ptr(k_cache), _ptr(v_cache),
+                                          _ptr(off, torch.int64), update_mode, _stream()),
+               "cake_decode_begin")
+        return k_cache, v_cache, off
+
+    def decode_step(self, layer: int, q_new, k_new, v_new, k_cache, v_cache) -> None:
+        _check(self.lib.cake_decode_step(self._h, layer, _ptr(q_new, self.dtype), _ptr(k_new, self.dtype),
+                                         _ptr(v_new, self.dtype), _ptr(k_cache), _ptr(v_cache),
+                                         _stream()), "cake_decode_step")
+
+    def decode_get_state(self, req: int, layer: int, length: int):
+        """(positions, scores, slots), each [H_kv][length], entries in ascending token position."""
+        H = self.cfg.n_kv_heads
+        pos = torch.empty(H, length, dtype=torch.int32, device="cuda")
+        sc = torch.empty(H, length, dtype=torch.float32, device="cuda")
+        sl = torch.empty(H, length, dtype=torch.int32, device="cuda")
+        _check(self.lib.cake_decode_get_state(self._h, req, layer, _ptr(pos), _ptr(sc), _ptr(sl),
+                                              _stream()), "cake_decode_get_state")
+        return pos, sc, sl
 
     def set_wait_limit(self, cycles: int) -> None:
         _check(self.lib.cake_set_wait_limit(self._h, cycles), "cake_set_wait_limit")

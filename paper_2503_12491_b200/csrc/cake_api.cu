@@ -67,6 +67,9 @@ void free_ctx(cake_ctx* c) {
   cudaFree(c->d_rowpart); cudaFree(c->d_colpart[0]); cudaFree(c->d_colpart[1]);
   cudaFree(c->d_tc_ops); cudaFree(c->d_tc_index); cudaFree(c->d_tc_sync);
   cudaFree(c->d_tc_rowpart); cudaFree(c->d_lse2_tc); cudaFree(c->d_hrow[0]); cudaFree(c->d_hrow[1]);
+  cudaFree(c->d_dec_off); cudaFree(c->d_dec_packed_off); cudaFree(c->d_dec_score); cudaFree(c->d_dec_pos);
+  cudaFree(c->d_dec_order); cudaFree(c->d_dec_meta);
+  if (c->h_budget_stage) cudaFreeHost(c->h_budget_stage);
   if (c->h_tc_ops) cudaFreeHost(c->h_tc_ops);
   if (c->h_tc_index) cudaFreeHost(c->h_tc_index);
   if (c->h_req) cudaFreeHost(c->h_req);
@@ -151,8 +154,9 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&x->n_sm, cudaDevAttrMultiProcessorCount, x->device);
   if (e != cudaSuccess) { free_ctx(x); return CAKE_ERR_CUDA; }
   {
-    // SMs left to the cascade kernels while a score kernel runs (CAKE_RESERVED_SMS, default 16)
-    int reserve = 16;
+    // SMs kept free of score CTAs (CAKE_RESERVED_SMS, default 0: the cascade kernels of the
+    // earlier layers fit beside a score CTA on the same SM)
+    int reserve = 0;
     if (const char* env = getenv("CAKE_RESERVED_SMS")) reserve = atoi(env);
     if (reserve < 0) reserve = 0;
     if (reserve > x->n_sm / 2) reserve = x->n_sm / 2;
@@ -248,6 +252,15 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
     ok = ok && dev_alloc(&x->d_hrow[0], (size_t)max_pairs * 128) == cudaSuccess;
     ok = ok && dev_alloc(&x->d_hrow[1], (size_t)max_pairs * 128) == cudaSuccess;
   }
+  // decode-time state: one slot per packed row plus one spare per (request, layer, head)
+  x->dec_rows_cap = x->pos_packed_cap + x->max_lists;
+  ok = ok && dev_alloc(&x->d_dec_off, (size_t)R * c.n_layers + 1) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_dec_packed_off, (size_t)R * c.n_layers + 1) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_dec_score, (size_t)x->dec_rows_cap) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_dec_pos, (size_t)x->dec_rows_cap) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_dec_order, (size_t)x->dec_rows_cap) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_dec_meta, (size_t)x->max_lists) == cudaSuccess;
+  ok = ok && cudaMallocHost((void**)&x->h_budget_stage, sizeof(int32_t) * R * c.n_layers) == cudaSuccess;
   ok = ok && cudaMemset(x->d_status, 0, sizeof(int32_t)) == cudaSuccess;
   ok = ok && cudaMemset(x->d_budget[0], 0, sizeof(int32_t) * R * c.n_layers) == cudaSuccess;
   ok = ok && cudaMemset(x->d_budget[1], 0, sizeof(int32_t) * R * c.n_layers) == cudaSuccess;
@@ -294,10 +307,9 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
     }
     const int32_t unit_keys = choose_unit_keys(T, c.n_kv_heads, ctx->n_sm);
     int32_t nu = 0, max_split = 0;
-    // the pooling / scatter kernels run on the SMs the score kernel leaves free: about two CTAs
-    // per such SM over all (request, head) pairs
-    const int reserve = ctx->n_sm - ctx->n_sm_score;
-    int want_split = (2 * (reserve > 0 ? reserve : 8)) / (n_req * c.n_kv_heads);
+    // the pooling / scatter kernels run one CTA per SM beside the score CTAs: about one CTA per
+    // SM over all (request, head) pairs
+    int want_split = ctx->n_sm / (n_req * c.n_kv_heads);
     if (want_split < 1) want_split = 1;
     int64_t list_off = 0, bound = 0;
     for (int r = 0; r < n_req; ++r) {
@@ -356,6 +368,7 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
   ctx->n_req = n_req;
   ctx->total_tokens = T;
   ctx->debug_epoch_skew = 0;
+  ctx->dec_ready = false;
   ctx->n_ind = ctx->n_pref = ctx->n_evicted = 0;
   ctx->alloc_of_buf[0] = ctx->alloc_of_buf[1] = -1;
   ctx->last_alloc = -1;
@@ -592,6 +605,69 @@ int32_t cake_profile_read(cake_ctx* ctx, double* ms_out, int64_t* spans_out, voi
 int32_t cake_uses_tensor_cores(const cake_ctx* ctx) {
   if (!ctx) return CAKE_ERR_ARG;
   return ctx->use_tc ? 1 : 0;
+}
+
+int64_t cake_decode_rows_bound(const cake_ctx* ctx) {
+  if (!ctx) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0) return CAKE_ERR_STATE;
+  return ctx->packed_rows_bound + (int64_t)ctx->n_req * ctx->cfg.n_layers * ctx->cfg.n_kv_heads;
+}
+
+int32_t cake_decode_begin(cake_ctx* ctx, const void* const* k_layers, const void* const* v_layers,
+                          void* k_cache, void* v_cache, int64_t* row_offsets_out, int32_t update_mode,
+                          void* stream) {
+  if (!ctx || ctx->n_req < 0) return ctx ? CAKE_ERR_STATE : CAKE_ERR_ARG;
+  const cake_config& c = ctx->cfg;
+  if (update_mode < CAKE_DECODE_ADD || update_mode > CAKE_DECODE_REPLACE) return CAKE_ERR_ARG;
+  if (ctx->n_evicted != c.n_layers || ctx->last_alloc != c.n_layers - 1) return CAKE_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  LayerPtrs ptrs;
+  memset(&ptrs, 0, sizeof(ptrs));
+  if (ctx->n_req > 0) {
+    if (!k_layers || !v_layers || !k_cache || !v_cache) return CAKE_ERR_ARG;
+    for (int l = 0; l < c.n_layers; ++l) {
+      if (!k_layers[l] || !v_layers[l]) return CAKE_ERR_ARG;
+      ptrs.k[l] = k_layers[l];
+      ptrs.v[l] = v_layers[l];
+    }
+  }
+  CAKE_CUDA_TRY(main_after_side(ctx, st));
+  // the step kernel's shared memory is sized from the largest head: read the final budgets back
+  ctx->dec_max_cap = 1;
+  if (ctx->n_req > 0) {
+    const size_t nb = sizeof(int32_t) * ctx->n_req * c.n_layers;
+    CAKE_CUDA_TRY(cudaMemcpyAsync(ctx->h_budget_stage, ctx->d_budget[(c.n_layers - 1) & 1], nb,
+                                  cudaMemcpyDeviceToHost, st));
+    CAKE_CUDA_TRY(cudaStreamSynchronize(st));
+    for (int i = 0; i < ctx->n_req * c.n_layers; ++i) {
+      const int64_t cap = (int64_t)ctx->h_budget_stage[i] + c.window + 1;
+      if (cap > ctx->dec_max_cap) ctx->dec_max_cap = cap;
+    }
+    const int G = c.n_q_heads / c.n_kv_heads;
+    if ((size_t)(G + 1) * ctx->dec_max_cap * sizeof(float) > 200 * 1024) return CAKE_ERR_CAPACITY;
+  }
+  const int32_t rc = launch_decode_begin(ctx, ptrs, k_cache, v_cache, row_offsets_out, st);
+  if (rc != CAKE_OK) return rc;
+  ctx->dec_update_mode = update_mode;
+  ctx->dec_ready = true;
+  return CAKE_OK;
+}
+
+int32_t cake_decode_step(cake_ctx* ctx, int32_t layer, const void* q_new, const void* k_new,
+                         const void* v_new, void* k_cache, void* v_cache, void* stream) {
+  if (!ctx || ctx->n_req < 0) return ctx ? CAKE_ERR_STATE : CAKE_ERR_ARG;
+  if (!ctx->dec_ready) return CAKE_ERR_STATE;
+  if (layer < 0 || layer >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
+  if (ctx->n_req > 0 && (!q_new || !k_new || !v_new || !k_cache || !v_cache)) return CAKE_ERR_ARG;
+  return launch_decode_step(ctx, layer, q_new, k_new, v_new, k_cache, v_cache, (cudaStream_t)stream);
+}
+
+int32_t cake_decode_get_state(cake_ctx* ctx, int32_t req, int32_t layer, int32_t* positions_out,
+                              float* scores_out, int32_t* slots_out, void* stream) {
+  if (!ctx) return CAKE_ERR_ARG;
+  if (ctx->n_req < 0 || !ctx->dec_ready) return CAKE_ERR_STATE;
+  if (req < 0 || req >= ctx->n_req || layer < 0 || layer >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
+  return launch_decode_read(ctx, req, layer, positions_out, scores_out, slots_out, (cudaStream_t)stream);
 }
 
 int32_t cake_set_wait_limit(cake_ctx* ctx, int64_t cycles) {

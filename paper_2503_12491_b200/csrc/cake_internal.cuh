@@ -156,6 +156,18 @@ struct cake_ctx {
   bool hhead_from_rows;    // entropy came from pass A (d_hrow) rather than from pass B partials
   int32_t n_tc_ctas, max_tc_segs, max_pairs;
   int32_t n_tc_waves;             // waves of the current plan
+  // ---- decode-time eviction (frozen budgets) ----
+  bool dec_ready;                 // cake_decode_begin has built the decode state of this batch
+  int32_t dec_update_mode;        // CAKE_DECODE_*
+  int64_t dec_max_cap;            // slots of the largest head of the batch (len + 1)
+  int64_t dec_rows_cap;           // capacity of the three arrays below
+  int64_t* d_dec_off;             // [max_requests*L + 1] decode row offsets
+  int64_t* d_dec_packed_off;      // [max_requests*L + 1] packed row offsets (set-up scratch)
+  float* d_dec_score;             // stored eviction score of every slot
+  int32_t* d_dec_pos;             // token position of every slot (-1: free)
+  int32_t* d_dec_order;           // per head: rank in ascending position -> slot
+  int4* d_dec_meta;               // [max_lists] (len, free slot, next position, frozen budget)
+  int32_t* h_budget_stage;        // pinned [max_requests*L] read-back of the final budgets
   int64_t wait_limit_cycles;      // bound of every device-side wait (0 = the default, about 2 s)
   int32_t debug_epoch_skew;       // test hook: added to the launch count the cross-CTA waits expect
   int32_t n_tc_asegs, n_tc_bsegs;          // pass-A / pass-B segments per layer
@@ -192,6 +204,13 @@ int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const v
 int32_t launch_pool(cake_ctx* ctx, int32_t layer, bool do_pool, bool finalize, cudaStream_t st);
 int32_t launch_allocate(cake_ctx* ctx, int32_t stage, cudaStream_t st);
 int32_t launch_evict(cake_ctx* ctx, int32_t stage, cudaStream_t st);
+// decode.cu
+int32_t launch_decode_begin(cake_ctx* ctx, const LayerPtrs& ptrs, void* k_cache, void* v_cache,
+                            int64_t* row_offsets, cudaStream_t st);
+int32_t launch_decode_step(cake_ctx* ctx, int32_t layer, const void* q_new, const void* k_new,
+                           const void* v_new, void* k_cache, void* v_cache, cudaStream_t st);
+int32_t launch_decode_read(cake_ctx* ctx, int32_t req, int32_t layer, int32_t* positions, float* scores,
+                           int32_t* slots, cudaStream_t st);
 // compact.cu
 int32_t launch_compact(cake_ctx* ctx, int32_t lo, int32_t hi, const LayerPtrs& ptrs, void* k_out,
                        void* v_out, int64_t* row_offsets, int32_t* positions, cudaStream_t st);

@@ -205,6 +205,17 @@ int32_t launch_compact(cake_ctx* ctx, int32_t lo, int32_t hi, const LayerPtrs& p
   return cuda_status(cudaGetLastError());
 }
 
+// Packed row offsets and positions of every layer into context scratch (decode-time set-up).
+int32_t run_sorted_positions_packed(cake_ctx* ctx, const int64_t* offsets_c, int32_t* out, cudaStream_t st) {
+  const cake_config& c = ctx->cfg;
+  int64_t* offsets = const_cast<int64_t*>(offsets_c);
+  const int32_t* budget = ctx->d_budget[(ctx->n_evicted - 1) & 1];
+  packed_offsets<<<1, 32, 0, st>>>(budget, offsets, ctx->n_req, c.n_layers, 0, c.n_layers, c.n_kv_heads,
+                                   c.window);
+  count_launch();
+  return run_sorted_positions(ctx, 0, ctx->n_req, 0, c.n_layers, offsets, out, 0, st);
+}
+
 int32_t launch_get_positions(cake_ctx* ctx, int32_t req, int32_t layer, int32_t* out,
                              int64_t capacity, cudaStream_t st) {
   if (capacity < 0) return CAKE_ERR_ARG;
