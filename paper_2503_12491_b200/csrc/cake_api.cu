@@ -154,9 +154,11 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&x->n_sm, cudaDevAttrMultiProcessorCount, x->device);
   if (e != cudaSuccess) { free_ctx(x); return CAKE_ERR_CUDA; }
   {
-    // SMs kept free of score CTAs (CAKE_RESERVED_SMS, default 0: the cascade kernels of the
-    // earlier layers fit beside a score CTA on the same SM)
-    int reserve = 0;
+    // SMs left to the cascade kernels while a score kernel runs (CAKE_RESERVED_SMS, default 16).
+    // The cascade kernels' CTAs are too large to share an SM with a score CTA, so they run on
+    // exactly these SMs and cannot slow a score CTA down: the score kernel's CTAs advance wave
+    // by wave together, and one delayed CTA delays all of them.
+    int reserve = 16;
     if (const char* env = getenv("CAKE_RESERVED_SMS")) reserve = atoi(env);
     if (reserve < 0) reserve = 0;
     if (reserve > x->n_sm / 2) reserve = x->n_sm / 2;
@@ -307,9 +309,10 @@ int32_t cake_begin(cake_ctx* ctx, int32_t n_req, const int64_t* cu, void* stream
     }
     const int32_t unit_keys = choose_unit_keys(T, c.n_kv_heads, ctx->n_sm);
     int32_t nu = 0, max_split = 0;
-    // the pooling / scatter kernels run one CTA per SM beside the score CTAs: about one CTA per
-    // SM over all (request, head) pairs
-    int want_split = ctx->n_sm / (n_req * c.n_kv_heads);
+    // the pooling / scatter kernels run on the SMs the score kernel leaves free: about two CTAs
+    // per such SM over all (request, head) pairs
+    const int reserve = ctx->n_sm - ctx->n_sm_score;
+    int want_split = (2 * (reserve > 0 ? reserve : 8)) / (n_req * c.n_kv_heads);
     if (want_split < 1) want_split = 1;
     int64_t list_off = 0, bound = 0;
     for (int r = 0; r < n_req; ++r) {

@@ -104,12 +104,7 @@ __device__ inline int block_excl_scan(int v, int* warp_tot, int* total) {
   return r;
 }
 
-// The cascade kernels run beside the score kernel of the following layers ON THE SAME SMs: a
-// score CTA leaves 8192 registers and about 26 KB of shared memory of its SM unused, and every
-// kernel below fits a CTA into that (256 threads of at most 32 registers, under 24 KB of shared
-// memory), so the score kernel can have every SM of the device.
-constexpr int kCoResidentCtasPerSm = 8;              // launch bound: 65536 / (256 * 8) = 32 registers
-constexpr int PH_THREADS = 256;
+constexpr int PH_THREADS = 1024;
 constexpr int PH_PER = 4;                            // consecutive tokens per thread and pass
 
 struct FinalizeArgs {        // preference of the layer from the tensor-core kernel's partials
@@ -186,7 +181,7 @@ __device__ void finalize_head(const FinalizeArgs& F, int req, int g, int hl, int
 // the layer's preference (tensor-core path).  The grid is small on purpose: it runs on the few
 // SMs the score kernel of the next layer leaves free.
 template <int R>
-__global__ void __launch_bounds__(PH_THREADS, kCoResidentCtasPerSm)
+__global__ void __launch_bounds__(PH_THREADS)
 pool_hist(const float* __restrict__ raw, float* __restrict__ fresh, const ReqInfo* __restrict__ reqs,
           uint32_t* __restrict__ hist, uint32_t* __restrict__ arrivals, int32_t* __restrict__ prefix,
           int n_split, int layer, int L, int Hkv, int64_t T, int kp, int mode, int do_pool,
@@ -466,7 +461,7 @@ __global__ void allocate_budgets(const double* __restrict__ dP, const ReqInfo* _
 
 // -------------------------------------------------------------------- evict
 constexpr int EV_THREADS = 256;
-constexpr int kTieCap = 1024;
+constexpr int kTieCap = 2048;
 
 struct EvictSmem {
   uint32_t hist[1024];
@@ -608,27 +603,19 @@ struct EvictArgs {
   int64_t T;
 };
 
-constexpr int SC_THREADS = 256;
+constexpr int SC_THREADS = 1024;
 constexpr int SC_PER = 4;
-
-// The per-bucket cursors of the scatter and the scratch of the threshold selection that the
-// list's last CTA runs afterwards are never live at the same time.
-union ScatterSmem {
-  uint32_t cnt[kBins];
-  EvictSmem ev;
-};
 
 // Newest layer of stage `stage`: one CTA per (split of a request's tokens, KV head, request)
 // scatters the pooled indicators into bucket order.  Only the buckets the layer's budget can
 // ever reach are stored (the budget never grows again, Proposition 1).  The CTA that completes
 // a list sets its threshold.
-__global__ void __launch_bounds__(SC_THREADS, kCoResidentCtasPerSm)
+__global__ void __launch_bounds__(SC_THREADS)
 scatter_new(const EvictArgs A) {
-  __shared__ ScatterSmem U;
-  __shared__ int s_warp_tot[32];
-  __shared__ int s_total;
+  __shared__ EvictSmem S;
+  __shared__ uint32_t s_cnt[kBins];
+  __shared__ uint32_t s_base[kBins];
   __shared__ int s_last;
-  uint32_t* const s_cnt = U.cnt;
   const int g = blockIdx.y, req = blockIdx.z;
   const ReqInfo rq = A.reqs[req];
   if ((int)blockIdx.x >= rq.nsplit) return;
@@ -643,8 +630,8 @@ scatter_new(const EvictArgs A) {
     less += __ldcg(&pf[i + 1]) < b ? 1 : 0;
     s_cnt[i] = 0;
   }
-  block_excl_scan(less, s_warp_tot, &s_total);
-  const int d_last = b > 0 ? min(s_total, kBins - 1) : -1;
+  block_excl_scan(less, S.warp_tot, &S.total);
+  const int d_last = b > 0 ? min(S.total, kBins - 1) : -1;
   __syncthreads();
   const float* src = A.fresh + (size_t)g * A.T + rq.cu;
   const int t0 = (int)blockIdx.x * rq.span, t1 = min(rq.n, t0 + rq.span);
@@ -669,11 +656,12 @@ scatter_new(const EvictArgs A) {
     if (run_len && run_bin >= 0) atomicAdd(&s_cnt[run_bin], run_len);
   }
   __syncthreads();
-  // reserve this split's range inside every bucket of the list; the count becomes the cursor
+  // reserve this split's range inside every bucket of the list
   uint32_t* gf = A.fill + (size_t)pair * kBins;
   for (int q = threadIdx.x; q < kBins; q += SC_THREADS) {
     const uint32_t c = s_cnt[q];
-    if (c) s_cnt[q] = (uint32_t)__ldcg(&pf[q]) + atomicAdd(&gf[q], c);
+    if (c) s_base[q] = (uint32_t)__ldcg(&pf[q]) + atomicAdd(&gf[q], c);
+    s_cnt[q] = 0;
   }
   __syncthreads();
   // pass 2: place the entries
@@ -702,7 +690,7 @@ scatter_new(const EvictArgs A) {
             if (bk[f] != run_bin) break;
             ++len;
           }
-          run_off = atomicAdd(&s_cnt[run_bin], len);
+          run_off = s_base[run_bin] + atomicAdd(&s_cnt[run_bin], len);
         }
       }
       if (run_bin >= 0) list[run_off++] = make_uint2(key[e], (uint32_t)(j0 + e));
@@ -719,13 +707,12 @@ scatter_new(const EvictArgs A) {
   __threadfence();
   for (int q = threadIdx.x; q < kBins; q += SC_THREADS) gf[q] = 0;       // ready for the next stage
   if (threadIdx.x == 0) A.arrivals[pair] = 0;
-  __syncthreads();                                  // the cursors are dead: their memory is reused
-  set_threshold(pf, list, b, -1, &A.states[lid], U.ev);
+  set_threshold(pf, list, b, -1, &A.states[lid], S);
 }
 
 // Older layers of stage `stage`: one CTA per (KV head, layer < stage, request) moves the list's
 // threshold to its new budget.
-__global__ void __launch_bounds__(EV_THREADS, kCoResidentCtasPerSm)
+__global__ void __launch_bounds__(EV_THREADS)
 thresholds_old(const EvictArgs A) {
   __shared__ EvictSmem S;
   const int g = blockIdx.x, layer = blockIdx.y, req = blockIdx.z;

@@ -333,9 +333,7 @@ __device__ __forceinline__ float4 merge_rows(float4 a, float4 b) {
 
 // ------------------------------------------------------------------ kernel
 template <int G, bool kEntropyB>
-// 112 registers per thread, not the 128 that one CTA per SM would allow: the 8192 registers left
-// over let a CTA of the cascade kernels run on the same SM (the kernel is no slower for it).
-__global__ void __maxnreg__(112)
+__global__ void __launch_bounds__(TC_THREADS, 1)
 score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                    const TcParams P) {
   extern __shared__ uint8_t smem_raw[];
