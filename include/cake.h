@@ -66,6 +66,14 @@ extern "C" {
 #define CAKE_IND_MEAN           1   /* Mean only                            */
 #define CAKE_IND_VAR            2   /* Var only                             */
 #define CAKE_IND_MEAN_TIMES_VAR 3   /* Mean * Var                           */
+#define CAKE_IND_WINDOW_SUM     4   /* sum over the window queries (S_w * Mean): the SnapKV
+                                       indicator of the paper's compatibility study,
+                                       Section 5.3, here under the preference allocation */
+/* How cake_allocate weighs the layers (Section 5.3, allocation ablation). */
+#define CAKE_ALLOC_PREFERENCE 0     /* P_l of Eq. 6 (the paper's method, default)          */
+#define CAKE_ALLOC_UNIFORM    1     /* every layer the same weight                         */
+#define CAKE_ALLOC_PYRAMID    2     /* weights falling linearly with the layer index:
+                                       w_l = 1 + s (L-1-2l)/(L-1), s = pyramid_slope        */
 
 /* How cake_decode_step combines a new token's pooled attention with a stored score (the
  * appendix listing calls it "update_score" without defining it). */
@@ -96,6 +104,10 @@ typedef struct cake_config {
   int64_t max_total_tokens; /* capacity: T = sum of prompt lengths per batch              */
   int32_t indicator_mode;   /* CAKE_IND_*: which combination of the window mean and
                                variance scores a key; gamma is used by mode 0 only        */
+  int32_t alloc_mode;       /* CAKE_ALLOC_*: what the budget split is proportional to; the
+                               rounding, the cap and the cascade are the same in every mode */
+  float   pyramid_slope;    /* s in [0, 1] for CAKE_ALLOC_PYRAMID (0 = uniform; 1 = the last
+                               layer gets no selectable budget)                            */
 } cake_config;
 
 /* Allocates a context (device state and scratch sized from the capacities) on

@@ -119,7 +119,7 @@ def layer_preference(a_obs: np.ndarray, tau1: float, tau2: float,
 # --------------------------------------------------------------------------
 # eviction indicator                                      (Section 4.3, Eq. 11)
 # --------------------------------------------------------------------------
-INDICATOR_KINDS = ("mean+var", "mean", "var", "mean*var")
+INDICATOR_KINDS = ("mean+var", "mean", "var", "mean*var", "sum")
 
 
 def indicator_raw(a_obs: np.ndarray, n_kv_heads: int, gamma: float,
@@ -144,6 +144,8 @@ def indicator_raw(a_obs: np.ndarray, n_kv_heads: int, gamma: float,
         return var
     if kind == "mean*var":
         return mean * var
+    if kind == "sum":                       # SnapKV's window sum (Section 5.3, compatibility study)
+        return abar.sum(axis=1)
     return mean + F64(gamma) * var
 
 
@@ -203,6 +205,46 @@ def webster(prefs: Sequence[float], seats: int) -> np.ndarray:
     order = np.lexsort((step[live], layer[live], -flat[live]))   # value desc, layer asc, s asc
     won = layer[live][order[:seats]]
     np.add.at(out, won, 1)
+    return out
+
+
+ALLOC_MODES = ("preference", "uniform", "pyramid")
+
+
+def allocation_weights(prefs: Sequence[float], n_layers: int, mode: str = "preference",
+                       slope: float = 0.0) -> np.ndarray:
+    """What the budget split of the layers seen so far is proportional to: the
+    preferences (Eq. 7 / Eq. 9), or one of the fixed patterns the paper's allocation
+    ablation compares with (Section 5.3): the same weight for every layer, or weights
+    falling linearly with the layer index, w_l = 1 + slope*(L-1-2l)/(L-1) (an arithmetic
+    progression with mean 1 over all L layers; slope in [0, 1])."""
+    assert mode in ALLOC_MODES
+    m1 = len(prefs)
+    if mode == "preference":
+        return np.asarray(prefs, dtype=F64)
+    if mode == "uniform" or n_layers <= 1:
+        return np.ones(m1, dtype=F64)
+    l = np.arange(m1, dtype=F64)
+    return F64(1.0) + F64(slope) * (F64(n_layers - 1) - 2.0 * l) / F64(n_layers - 1)
+
+
+def cumulative_attention(q_all: np.ndarray, k: np.ndarray) -> np.ndarray:
+    """H2O's indicator: the attention every key has received from ALL prompt queries
+    (causal softmax rows summed over the queries), averaged over the group's query heads.
+    q_all: [H_q][N][d], k: [H_kv][N][d] -> [H_kv][N].  It needs the whole prefill
+    attention and is not computed by the window-score path; a caller that has it hands it
+    to the cascade in place of Eq. 11's indicator (Section 5.3, compatibility study)."""
+    q = np.asarray(q_all, dtype=F64)
+    kk = np.asarray(k, dtype=F64)
+    Hq, N, d = q.shape
+    Hkv = kk.shape[0]
+    G = Hq // Hkv
+    out = np.zeros((Hkv, N), dtype=F64)
+    mask = np.triu(np.ones((N, N), dtype=bool), 1)
+    for h in range(Hq):
+        s = q[h] @ kk[h // G].T / np.sqrt(F64(d))
+        s[mask] = -np.inf
+        out[h // G] += softmax_rows(s).sum(axis=0) / G
     return out
 
 

@@ -46,6 +46,7 @@ class CakeConfig(ctypes.Structure):
         ("tau1", ctypes.c_float), ("tau2", ctypes.c_float),
         ("total_budget", ctypes.c_int64), ("max_requests", ctypes.c_int32),
         ("max_total_tokens", ctypes.c_int64), ("indicator_mode", ctypes.c_int32),
+        ("alloc_mode", ctypes.c_int32), ("pyramid_slope", ctypes.c_float),
     ]
 
 
@@ -159,13 +160,14 @@ class Cake:
                  window: int, pool_kernel: int, gamma: float, total_budget: int,
                  max_requests: int, max_total_tokens: int, dtype: torch.dtype = torch.bfloat16,
                  tau1: float = 1.0, tau2: float = 1.0, pool_mode: int = CAKE_POOL_MAX,
-                 var_ddof: int = 0, indicator_mode: int = 0):
+                 var_ddof: int = 0, indicator_mode: int = 0, alloc_mode: int = 0,
+                 pyramid_slope: float = 0.0):
         self.lib = load_library()
         self.cfg = CakeConfig(n_layers, n_q_heads, n_kv_heads, head_dim, window, pool_kernel,
                               pool_mode, var_ddof,
                               CAKE_DTYPE_FP32 if dtype == torch.float32 else CAKE_DTYPE_BF16,
                               gamma, tau1, tau2, total_budget, max_requests, max_total_tokens,
-                              indicator_mode)
+                              indicator_mode, alloc_mode, pyramid_slope)
         self.dtype = dtype
         self._h = ctypes.c_void_p()
         _check(self.lib.cake_create(ctypes.byref(self.cfg), ctypes.byref(self._h)), "cake_create")

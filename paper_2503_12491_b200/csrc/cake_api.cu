@@ -136,7 +136,9 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   if (c.var_ddof != 0 && !(c.var_ddof == 1 && c.window >= 2)) return CAKE_ERR_ARG;
   if (c.dtype != CAKE_DTYPE_FP32 && c.dtype != CAKE_DTYPE_BF16) return CAKE_ERR_ARG;
   if (!(c.tau1 > 0.f) || !(c.tau2 > 0.f) || !std::isfinite(c.gamma)) return CAKE_ERR_ARG;
-  if (c.indicator_mode < CAKE_IND_MEAN_PLUS_VAR || c.indicator_mode > CAKE_IND_MEAN_TIMES_VAR) return CAKE_ERR_ARG;
+  if (c.indicator_mode < CAKE_IND_MEAN_PLUS_VAR || c.indicator_mode > CAKE_IND_WINDOW_SUM) return CAKE_ERR_ARG;
+  if (c.alloc_mode < CAKE_ALLOC_PREFERENCE || c.alloc_mode > CAKE_ALLOC_PYRAMID) return CAKE_ERR_ARG;
+  if (c.alloc_mode == CAKE_ALLOC_PYRAMID && !(c.pyramid_slope >= 0.f && c.pyramid_slope <= 1.f)) return CAKE_ERR_ARG;
   if (c.max_requests < 1 || c.max_total_tokens < 1) return CAKE_ERR_ARG;
   if (c.max_total_tokens > ((int64_t)1 << 31) - 1024) return CAKE_ERR_ARG;
   if (c.total_budget < (int64_t)c.n_layers * c.window) return CAKE_ERR_BUDGET;

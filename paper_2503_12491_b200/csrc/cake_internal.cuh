@@ -219,10 +219,12 @@ int32_t launch_get_positions(cake_ctx* ctx, int32_t req, int32_t layer, int32_t*
 
 // The eviction indicator of one key from the mean and variance of its window attention
 // (Section 4.3, Eq. 11, and the combinations of the paper's indicator ablation).
-__device__ __forceinline__ float combine_indicator(int mode, float gamma, float mean, float var) {
+__device__ __forceinline__ float combine_indicator(int mode, float gamma, float mean, float var,
+                                                   float sw) {
   return mode == CAKE_IND_MEAN_PLUS_VAR ? fmaf(gamma, var, mean)
          : mode == CAKE_IND_MEAN        ? mean
          : mode == CAKE_IND_VAR         ? var
+         : mode == CAKE_IND_WINDOW_SUM  ? mean * sw
                                         : mean * var;
 }
 

@@ -319,7 +319,8 @@ constexpr int kMaxCand = 1024;
 // threshold is found by bisection over the bit patterns of the doubles.
 __global__ void allocate_budgets(const double* __restrict__ dP, const ReqInfo* __restrict__ reqs,
                                  const int32_t* __restrict__ prev, int32_t* __restrict__ cur,
-                                 int32_t* __restrict__ status, int stage, int L, int64_t seats) {
+                                 int32_t* __restrict__ status, int stage, int L, int64_t seats,
+                                 int alloc_mode, double slope) {
   __shared__ double sP[CAKE_MAX_LAYERS];
   __shared__ int64_t s_lo[CAKE_MAX_LAYERS];
   __shared__ int32_t s_off[CAKE_MAX_LAYERS + 1];
@@ -337,7 +338,11 @@ __global__ void allocate_budgets(const double* __restrict__ dP, const ReqInfo* _
   bool bad = false;
   bool anypos = false;
   for (int l = lane; l < La; l += 32) {
-    const double p = dP[(size_t)req * L + l];
+    // what the split is proportional to: the preference (Eq. 7 / Eq. 9), or one of the fixed
+    // patterns of the paper's allocation ablation (Section 5.3)
+    double p = dP[(size_t)req * L + l];
+    if (alloc_mode == CAKE_ALLOC_UNIFORM) p = 1.0;
+    else if (alloc_mode == CAKE_ALLOC_PYRAMID) p = L > 1 ? 1.0 + slope * (double)(L - 1 - 2 * l) / (double)(L - 1) : 1.0;
     sP[l] = p;
     if (!(p >= 0.0) || isinf(p)) bad = true;
     if (p > 0.0) anypos = true;
@@ -783,7 +788,8 @@ int32_t launch_allocate(cake_ctx* ctx, int32_t stage, cudaStream_t st) {
   if (ctx->n_req == 0) return CAKE_OK;
   allocate_budgets<<<ctx->n_req, 32, 0, st>>>(ctx->d_P, ctx->d_req, ctx->d_budget[(stage + 1) & 1],
                                               ctx->d_budget[stage & 1], ctx->d_status, stage,
-                                              c.n_layers, ctx->sel_budget);
+                                              c.n_layers, ctx->sel_budget, c.alloc_mode,
+                                              (double)c.pyramid_slope);
   count_launch();
   return cuda_status(cudaGetLastError());
 }

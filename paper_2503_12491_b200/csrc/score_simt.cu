@@ -289,7 +289,7 @@ score_colstats_simt(const T* __restrict__ q_win, const T* __restrict__ k,
     if (valid && q4 == 0) {
       const float mean = a1 * inv_sw;
       const float var = fmaxf(a2 * inv_sw - mean * mean, 0.f) * bessel;
-      raw[(size_t)g * T_tokens + rq.cu + key0 + key_l] = combine_indicator(ind_mode, gamma, mean, var);
+      raw[(size_t)g * T_tokens + rq.cu + key0 + key_l] = combine_indicator(ind_mode, gamma, mean, var, (float)Sw);
 #pragma unroll
       for (int h = 0; h < 8; ++h) {
         if (h < G) {

@@ -70,6 +70,7 @@ struct TcParams {
   uint32_t* pair_cnt;           // [pairs] delivered pass-A partials (monotonic over layers)
   uint32_t* pair_done;          // [pairs] merged rows (monotonic over layers); null = pass B only
   float* lse2;                  // [pair][128] in tile row order r' = i*G + h
+  const float* lse_ext;         // caller's natural-log LSE [req][H_q][S_w], or null
   float4* rowpart;              // pass A out: [A-segment][group][128] (m, z_all, z_win, w)
   float* raw;                   // pass B out: [H_kv][T]
   float* colpart;               // pass B out: [B-segment][statistics warp][G][2]
@@ -658,7 +659,19 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       }
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
-      const float4 v = __ldcg(reinterpret_cast<const float4*>(P.lse2 + (size_t)pair * 128) + lane);
+      float4 v;
+      if (P.lse_ext) {
+        // the caller's natural-log values [req][H_q][S_w]: tile row r' = i*G + h, base 2
+        float x[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int r = 4 * lane + e, i = r / G, h = r - i * G;
+          x[e] = r < P.rows ? __ldg(&P.lse_ext[((size_t)op.req * P.Hq + op.g * G + h) * P.Sw + i]) * kLog2e : 0.f;
+        }
+        v = make_float4(x[0], x[1], x[2], x[3]);
+      } else {
+        v = __ldcg(reinterpret_cast<const float4*>(P.lse2 + (size_t)pair * 128) + lane);
+      }
       // stored negated: the statistics warps add them
       reinterpret_cast<float4*>(S.lse + slot * 128)[lane] = make_float4(-v.x, -v.y, -v.z, -v.w);
       __syncwarp();
@@ -787,7 +800,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
             const float mean = a1 * inv_g * inv_sw;
             const float var = fmaxf(a2 * inv_g * inv_g * inv_sw - mean * mean, 0.f) * P.bessel;
-            P.raw[op.base + j] = combine_indicator(P.ind_mode, P.gamma, mean, var);
+            P.raw[op.base + j] = combine_indicator(P.ind_mode, P.gamma, mean, var, (float)P.Sw);
           }
         }
         __syncwarp();
@@ -927,16 +940,6 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512)
                  : "memory");
   }
-}
-
-// External natural-log LSE [req][H_q][S_w] -> base-2, tile row order.
-__global__ void tc_lse_permute(const float* __restrict__ lse, float* __restrict__ lse2, int Hkv, int G,
-                               int Sw) {
-  const int req = blockIdx.x, g = blockIdx.y, r = threadIdx.x;
-  if (r >= G * Sw) return;
-  const int i = r / G, h = r - i * G;
-  lse2[((size_t)req * Hkv + g) * 128 + r] =
-      lse[((size_t)req * Hkv * G + g * G + h) * Sw + i] * kLog2e;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -1231,6 +1234,7 @@ int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const v
   P.pair_aseg = ctx->d_tc_index;
   P.pair_cnt = ctx->d_tc_sync;
   P.lse2 = ctx->d_lse2_tc;
+  P.lse_ext = lse;
   P.rowpart = ctx->d_tc_rowpart;
   P.raw = ctx->d_raw[layer & 1];
   P.colpart = ctx->d_colpart[layer & 1];
@@ -1250,9 +1254,6 @@ int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const v
   const int32_t* cta_full = ctx->d_tc_index + 2 * (n_pairs + 1);
   if (lse) {
     // denominators supplied: pass B alone, entropy from its columns
-    const dim3 pairs(ctx->n_req, c.n_kv_heads);
-    tc_lse_permute<<<pairs, 128, 0, st>>>(lse, ctx->d_lse2_tc, c.n_kv_heads, G, c.window);
-    count_launch();
     ctx->hhead_from_rows = false;
     P.cta_op = cta_full + (ctx->n_sm + 1);
     P.pair_done = nullptr;

@@ -183,3 +183,79 @@ def test_a_wait_that_runs_out_returns_a_status_and_the_context_recovers():
     assert torch.equal(got[2], want[2]) and torch.equal(got[3][:n], want[3][:n])
     assert torch.equal(got[0][:n], want[0][:n]) and torch.equal(got[1][:n], want[1][:n])
     cake.destroy()
+
+
+# ------------------------------------------------ variants of the paper's comparison study
+@pytest.mark.parametrize("make,tc", [(bf16_case, True), (fp32_case, False)])
+def test_window_sum_indicator(make, tc):
+    """The SnapKV indicator (sum of the window queries' attention) under the preference
+    allocation (Section 5.3, compatibility study)."""
+    check_scores(make(), cake_kw=dict(indicator_mode=4), oracle_kw=dict(indicator="sum"), expect_tc=tc)
+
+
+@pytest.mark.parametrize("mode,name,slope", [(1, "uniform", 0.0), (2, "pyramid", 0.6), (2, "pyramid", 1.0)])
+def test_uniform_and_pyramid_allocation_bit_exact(mode, name, slope):
+    """The fixed allocation patterns of the allocation ablation (Section 5.3) through the same
+    rounding, cap and cascade: budgets of every stage and the final retained sets."""
+    L = 6
+    w = fp32_case(n_layers=L, seq_lens=(400, 90), total_budget=L * 16 + 333)
+    qs, ks, vs = harness.device_inputs(w)
+    cake = harness.cake_for(w, alloc_mode=mode, pyramid_slope=slope)
+    cake.begin(w.cu_seqlens)
+    cu = w.cu_seqlens
+    inds = []
+    for l in range(L):
+        cake.score_layer(l, qs[l], ks[l])
+        inds.append(cake.get_indicators(l).cpu().numpy())
+        cake.allocate(l)
+        got = cake.get_budgets().cpu().numpy()
+        for r, N in enumerate(w.seq_lens):
+            wts = O.allocation_weights([0.0] * (l + 1), L, name, slope)
+            want = O.stage_budgets(wts, w.total_budget, L, w.window, N) + w.window
+            assert np.array_equal(got[r, :l + 1], want), (l, r, got[r], want)
+        cake.evict(l)
+    budgets = cake.get_budgets().cpu().numpy()
+    for r, N in enumerate(w.seq_lens):
+        n = N - w.window
+        wts = O.allocation_weights([0.0] * L, L, name, slope)
+        c = O.cascade([inds[l][:, cu[r]:cu[r] + n].astype(np.float64) for l in range(L)], wts,
+                      total_budget=w.total_budget, window=w.window, seq_len=N)
+        assert np.array_equal(budgets[r], c.budgets)
+        for l in range(L):
+            got_pos = cake.get_positions(r, l, int(budgets[r, l])).cpu().numpy()
+            for g in range(w.n_kv_heads):
+                assert np.array_equal(got_pos[g], c.positions[l][g])
+    assert cake.status() == 0
+    cake.destroy()
+
+
+def test_cumulative_attention_indicator_through_the_hook():
+    """H2O's cumulative attention needs the whole prefill attention, which the window-score path
+    does not compute: a caller that has it hands it over with cake_set_indicators and gets the
+    preference allocation and the cascade on it (Section 5.3, compatibility study)."""
+    L = 3
+    w = fp32_case(n_layers=L, seq_lens=(260,), total_budget=L * 16 + 150)
+    qs, ks, vs = harness.device_inputs(w)
+    N, n = w.seq_lens[0], w.seq_lens[0] - w.window
+    rng = np.random.default_rng(9)
+    cake = harness.cake_for(w)
+    cake.begin(w.cu_seqlens)
+    P = np.array([[1.5, 0.4, 2.2]])
+    cake.set_preferences(torch.from_numpy(P).cuda())
+    inds = []
+    for l in range(L):
+        q_all = rng.normal(size=(w.n_q_heads, N, w.head_dim))     # stands in for the prompt's queries
+        ind = O.cumulative_attention(q_all, to_np(ks[l]))[:, :N].astype(np.float32)
+        inds.append(ind)
+        cake.set_indicators(l, torch.from_numpy(ind).cuda())
+        cake.allocate(l)
+        cake.evict(l)
+    budgets = cake.get_budgets().cpu().numpy()
+    c = O.cascade([x[:, :n].astype(np.float64) for x in inds], P[0], total_budget=w.total_budget,
+                  window=w.window, seq_len=N)
+    assert np.array_equal(budgets[0], c.budgets)
+    for l in range(L):
+        got = cake.get_positions(0, l, int(budgets[0, l])).cpu().numpy()
+        for g in range(w.n_kv_heads):
+            assert np.array_equal(got[g], c.positions[l][g])
+    cake.destroy()

@@ -33,11 +33,13 @@ def test_library_builds_loads_and_exports_everything():
 
 
 def test_config_struct_matches_header_layout():
-    # 9 int32, 3 float, int64, int32 (+pad), int64, int32 (+pad)
-    assert ctypes.sizeof(binding.CakeConfig) == 80
+    # 9 int32, 3 float, int64, int32 (+pad), int64, 2 int32, float (+pad)
+    assert ctypes.sizeof(binding.CakeConfig) == 88
     assert binding.CakeConfig.total_budget.offset == 48
     assert binding.CakeConfig.max_total_tokens.offset == 64
     assert binding.CakeConfig.indicator_mode.offset == 72
+    assert binding.CakeConfig.alloc_mode.offset == 76
+    assert binding.CakeConfig.pyramid_slope.offset == 80
 
 
 def test_argument_errors_need_no_gpu():
@@ -50,7 +52,11 @@ def test_argument_errors_need_no_gpu():
     assert lib.cake_create(ctypes.byref(small), ctypes.byref(h)) == binding.CAKE_ERR_BUDGET
     even = binding.CakeConfig(4, 4, 4, 64, 16, 4, 0, 0, 0, 1.0, 1.0, 1.0, 512, 1, 512)  # even kernel
     assert lib.cake_create(ctypes.byref(even), ctypes.byref(h)) == binding.CAKE_ERR_ARG
-    mode = binding.CakeConfig(4, 4, 4, 64, 16, 5, 0, 0, 0, 1.0, 1.0, 1.0, 512, 1, 512, 4)  # no such indicator
+    mode = binding.CakeConfig(4, 4, 4, 64, 16, 5, 0, 0, 0, 1.0, 1.0, 1.0, 512, 1, 512, 5)  # no such indicator
     assert lib.cake_create(ctypes.byref(mode), ctypes.byref(h)) == binding.CAKE_ERR_ARG
+    alloc = binding.CakeConfig(4, 4, 4, 64, 16, 5, 0, 0, 0, 1.0, 1.0, 1.0, 512, 1, 512, 0, 3)  # no such allocation
+    assert lib.cake_create(ctypes.byref(alloc), ctypes.byref(h)) == binding.CAKE_ERR_ARG
+    slope = binding.CakeConfig(4, 4, 4, 64, 16, 5, 0, 0, 0, 1.0, 1.0, 1.0, 512, 1, 512, 0, 2, 1.5)
+    assert lib.cake_create(ctypes.byref(slope), ctypes.byref(h)) == binding.CAKE_ERR_ARG
     assert lib.cake_begin(None, 0, None, None) == binding.CAKE_ERR_ARG
     assert lib.cake_allocate(None, 0, None) == binding.CAKE_ERR_ARG

@@ -632,3 +632,54 @@ def test_decode_init_takes_the_survivors_indicators():
         assert np.array_equal(heads[g].positions, positions[g])
         assert np.array_equal(heads[g].scores, ind[g][positions[g][:6]])
         assert np.array_equal(heads[g].k, k[g][positions[g]])
+
+
+# --------------------------------------------- variants of the comparison study
+def test_window_sum_indicator_is_the_mean_times_the_window():
+    rng = np.random.default_rng(41)
+    q, k = rand_case(rng, Hq=4, Hkv=2, Sw=5, N=13)
+    obs = O.observed_attention(q, k)
+    tot = O.indicator_raw(obs, 2, gamma=7.0, kind="sum")
+    assert np.allclose(tot, 5 * O.indicator_raw(obs, 2, gamma=7.0, kind="mean"), rtol=1e-13)
+    for g in range(2):
+        for j in range(obs.shape[2]):
+            want = sum(obs[2 * g + h, i, j] for h in range(2) for i in range(5)) / 2
+            assert math.isclose(tot[g, j], want, rel_tol=1e-12)
+
+
+def test_allocation_weights_of_the_ablation():
+    P = [0.3, 2.0, 1.1, 0.7]
+    assert np.array_equal(O.allocation_weights(P, 8, "preference"), P)
+    assert np.array_equal(O.allocation_weights(P, 8, "uniform"), np.ones(4))
+    w = O.allocation_weights([0] * 8, 8, "pyramid", slope=0.5)
+    assert np.allclose(np.diff(w), -2 * 0.5 / 7)                 # arithmetic progression
+    assert math.isclose(w.mean(), 1.0, rel_tol=1e-15) and math.isclose(w[0], 1.5) and math.isclose(w[-1], 0.5)
+    assert np.array_equal(O.allocation_weights([0] * 3, 8, "pyramid", slope=0.5), w[:3])   # seen layers only
+    assert O.allocation_weights([0] * 8, 8, "pyramid", slope=1.0)[-1] == 0.0
+    assert np.array_equal(O.allocation_weights([5.0], 1, "pyramid", slope=0.7), [1.0])
+    # uniform weights give equal budgets (the remainder to the first layers), pyramid never
+    # gives a later layer more, and both keep Proposition 1 (fixed weights)
+    b = O.stage_budgets(O.allocation_weights([0] * 5, 8, "uniform"), 8 * 4 + 103, 8, 4, 1000)
+    assert b.sum() == 103 and b.max() - b.min() <= 1 and np.all(np.diff(b) <= 0)
+    prev = None
+    for m in range(8):
+        b = O.stage_budgets(O.allocation_weights([0] * (m + 1), 8, "pyramid", 0.8), 8 * 4 + 500, 8, 4, 10000)
+        assert b.sum() == 500 and np.all(np.diff(b) <= 0)
+        if prev is not None:
+            assert np.all(b[:-1] <= prev)
+        prev = b
+
+
+def test_cumulative_attention_brute_force():
+    rng = np.random.default_rng(42)
+    Hq, Hkv, N, d = 4, 2, 7, 8
+    q, k = rng.normal(size=(Hq, N, d)), rng.normal(size=(Hkv, N, d))
+    got = O.cumulative_attention(q, k)
+    want = np.zeros((Hkv, N))
+    for h in range(Hq):
+        for i in range(N):
+            e = [math.exp(sum(q[h, i, t] * k[h // 2, j, t] for t in range(d)) / math.sqrt(d)) for j in range(i + 1)]
+            for j in range(i + 1):
+                want[h // 2, j] += e[j] / sum(e) / 2
+    assert np.allclose(got, want, rtol=1e-12)
+    assert np.allclose(got.sum(axis=1), N)          # every query row sums to one
