@@ -179,6 +179,30 @@ int32_t cake_compact(cake_ctx* ctx, int32_t layer_lo, int32_t layer_hi,
                      void* k_out, void* v_out, int64_t* row_offsets_out,
                      int32_t* positions_out, void* stream);
 
+/* cake_compact with 4-bit output: the retained rows written as asymmetric INT4 codes, keys
+ * quantised per channel and values per token -- the combination of eviction and KIVI-style
+ * quantisation the paper evaluates (Appendix "Comparison and Compatibility with Quantization
+ * Methods").  Same packed row order, row offsets and positions as cake_compact.
+ *   A group of `group` (32, 64 or 128, at most d) values shares zero = min and
+ *   scale = (max - min) / 15 (1 when max = min); code = clamp(rint((x - zero) / scale), 0, 15)
+ *   in IEEE fp32; x is recovered as zero + code * scale.
+ *   values: groups of `group` consecutive channels of a row.
+ *           v_codes uint8 [rows][d/2] (even channel in the low nibble),
+ *           v_scale, v_zero fp32 [rows][d/group]
+ *   keys:   one group per channel over `group` consecutive packed rows of a (request, layer,
+ *           head); the last group of a head may be shorter.
+ *           k_codes uint8 [rows][d/2]; k_scale, k_zero fp32 [key groups][d], where block
+ *           (r,l) owns the key groups kgroup_offsets[r*L+l] .. kgroup_offsets[r*L+l+1]-1,
+ *           laid out [H_kv][ceil(len/group)]
+ *   kgroup_offsets_out: device int64 [n_req*L + 1].
+ * Capacities: rows <= cake_packed_rows_bound(); key groups <= rows / group + n_req*L*H_kv. */
+int32_t cake_compact_int4(cake_ctx* ctx, int32_t layer_lo, int32_t layer_hi,
+                          const void* const* k_layers, const void* const* v_layers, int32_t group,
+                          uint8_t* k_codes, float* k_scale, float* k_zero,
+                          uint8_t* v_codes, float* v_scale, float* v_zero,
+                          int64_t* row_offsets_out, int64_t* kgroup_offsets_out,
+                          int32_t* positions_out, void* stream);
+
 /* Upper bound on the rows cake_compact writes for the current batch:
  * H_kv * sum_r min(B_total, L*N_r).  Returns the bound or a negative error. */
 int64_t cake_packed_rows_bound(const cake_ctx* ctx);

@@ -349,6 +349,57 @@ def compact(k: np.ndarray, v: np.ndarray, positions: Sequence[np.ndarray]
 
 
 # --------------------------------------------------------------------------
+# quantised compaction       (Appendix "Comparison and Compatibility with
+#                             Quantization Methods": KIVI-INT4 with CAKE)
+# --------------------------------------------------------------------------
+# Asymmetric 4-bit codes of the compacted rows, keys per channel and values per
+# token.  The code is an integer decided by floating point, so the arithmetic is
+# fixed: IEEE float32, zero = min, scale = (max - min)/15 (1 if max = min),
+# code = clip(rint((x - zero)/scale), 0, 15) with round-half-to-even.
+F32 = np.float32
+
+
+def int4_codes(x: np.ndarray, axis: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Codes (uint8, 0..15), scale and zero (float32, `axis` kept with length 1) of one
+    group spanning `axis`."""
+    x = np.asarray(x, dtype=F32)
+    zero = x.min(axis=axis, keepdims=True)
+    span = (x.max(axis=axis, keepdims=True) - zero).astype(F32)
+    scale = np.where(span > 0, (span / F32(15.0)).astype(F32), F32(1.0)).astype(F32)
+    q = np.rint(((x - zero).astype(F32) / scale).astype(F32))
+    return np.clip(q, 0, 15).astype(np.uint8), scale, zero
+
+
+def quantize_values_per_token(v_rows: np.ndarray, group: int):
+    """v_rows [rows][d] -> codes [rows][d], scale, zero [rows][d/group]: groups of
+    `group` consecutive channels of a row."""
+    rows, d = v_rows.shape
+    x = np.asarray(v_rows, dtype=F32).reshape(rows, d // group, group)
+    q, s, z = int4_codes(x, axis=2)
+    return q.reshape(rows, d), s[..., 0], z[..., 0]
+
+
+def quantize_keys_per_channel(k_rows: np.ndarray, group: int):
+    """k_rows [len][d] (one head's compacted rows) -> codes [len][d], scale, zero
+    [ceil(len/group)][d]: per channel, groups of `group` consecutive rows (the last
+    group may be shorter)."""
+    n, d = k_rows.shape
+    codes = np.zeros((n, d), dtype=np.uint8)
+    scales, zeros = [], []
+    for t0 in range(0, n, group):
+        q, s, z = int4_codes(np.asarray(k_rows[t0:t0 + group], dtype=F32), axis=0)
+        codes[t0:t0 + group] = q
+        scales.append(s[0])
+        zeros.append(z[0])
+    return codes, np.array(scales, dtype=F32).reshape(-1, d), np.array(zeros, dtype=F32).reshape(-1, d)
+
+
+def pack_nibbles(codes: np.ndarray) -> np.ndarray:
+    """[rows][d] codes -> [rows][d/2] bytes, the even channel in the low nibble."""
+    return (codes[:, 0::2] | (codes[:, 1::2] << 4)).astype(np.uint8)
+
+
+# --------------------------------------------------------------------------
 # decode-time eviction        (Section 5.1 "Implementation Details"; Appendix
 #                              "More Implementation Details"; Listing 1, the
 #                              branches taken when not prefilling)

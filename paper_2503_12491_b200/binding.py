@@ -31,6 +31,7 @@ EXPORTS = [
     "cake_profile_enable", "cake_profile_read", "cake_uses_tensor_cores",
     "cake_select_positions_static", "cake_plan_info", "cake_set_wait_limit", "cake_debug_skew_sync",
     "cake_decode_rows_bound", "cake_decode_begin", "cake_decode_step", "cake_decode_get_state",
+    "cake_compact_int4",
 ]
 PROF_KINDS = ["score", "finalize", "allocate", "evict", "compact"]
 
@@ -75,6 +76,8 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.cake_allocate.argtypes = [vp, i32, vp]
     lib.cake_evict.argtypes = [vp, i32, vp]
     lib.cake_compact.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, vp, vp, vp, vp]
+    lib.cake_compact_int4.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), i32,
+                                      vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.cake_packed_rows_bound.argtypes = [vp]
     lib.cake_packed_rows_bound.restype = i64
     lib.cake_get_indicators.argtypes = [vp, i32, vp, vp]
@@ -237,6 +240,29 @@ class Cake:
                                      _ptr(row_offsets, torch.int64), _ptr(positions, torch.int32),
                                      _stream()), "cake_compact")
         return k_out, v_out, row_offsets, positions
+
+    def compact_int4(self, k_layers, v_layers, group: int = 32):
+        """cake_compact_int4 over all layers; returns a dict of the output tensors."""
+        L, d = self.cfg.n_layers, self.cfg.head_dim
+        dev = torch.device("cuda", torch.cuda.current_device())
+        rows = max(self.packed_rows_bound(), 1)
+        kg = rows // group + self.n_req * L * self.cfg.n_kv_heads + 1
+        out = dict(k_codes=torch.zeros(rows, d // 2, dtype=torch.uint8, device=dev),
+                   k_scale=torch.zeros(kg, d, dtype=torch.float32, device=dev),
+                   k_zero=torch.zeros(kg, d, dtype=torch.float32, device=dev),
+                   v_codes=torch.zeros(rows, d // 2, dtype=torch.uint8, device=dev),
+                   v_scale=torch.zeros(rows, d // group, dtype=torch.float32, device=dev),
+                   v_zero=torch.zeros(rows, d // group, dtype=torch.float32, device=dev),
+                   row_offsets=torch.empty(self.n_req * L + 1, dtype=torch.int64, device=dev),
+                   kgroup_offsets=torch.empty(self.n_req * L + 1, dtype=torch.int64, device=dev),
+                   positions=torch.empty(rows, dtype=torch.int32, device=dev))
+        kp = (ctypes.c_void_p * L)(*[_ptr(t, self.dtype) for t in k_layers])
+        vp = (ctypes.c_void_p * L)(*[_ptr(t, self.dtype) for t in v_layers])
+        _check(self.lib.cake_compact_int4(
+            self._h, 0, L, kp, vp, group, _ptr(out["k_codes"]), _ptr(out["k_scale"]), _ptr(out["k_zero"]),
+            _ptr(out["v_codes"]), _ptr(out["v_scale"]), _ptr(out["v_zero"]), _ptr(out["row_offsets"]),
+            _ptr(out["kgroup_offsets"]), _ptr(out["positions"]), _stream()), "cake_compact_int4")
+        return out
 
     # -- getters / hooks
     def get_indicators(self, layer: int) -> torch.Tensor:

@@ -17,7 +17,7 @@ INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG, "libcake.so")
 
 SOURCES = ["cake_api.cu", "score_simt.cu", "score_tc.cu", "cascade.cu", "compact.cu",
-           "decode.cu", "select_static.cu"]
+           "decode.cu", "quant.cu", "select_static.cu"]
 
 
 def _nvcc() -> str:

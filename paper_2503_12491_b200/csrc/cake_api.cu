@@ -474,6 +474,38 @@ int32_t cake_compact(cake_ctx* ctx, int32_t layer_lo, int32_t layer_hi, const vo
   return rc;
 }
 
+int32_t cake_compact_int4(cake_ctx* ctx, int32_t layer_lo, int32_t layer_hi, const void* const* k_layers,
+                          const void* const* v_layers, int32_t group, uint8_t* k_codes, float* k_scale,
+                          float* k_zero, uint8_t* v_codes, float* v_scale, float* v_zero,
+                          int64_t* row_offsets_out, int64_t* kgroup_offsets_out, int32_t* positions_out,
+                          void* stream) {
+  if (!ctx || ctx->n_req < 0) return ctx ? CAKE_ERR_STATE : CAKE_ERR_ARG;
+  const cake_config& c = ctx->cfg;
+  if (layer_lo < 0 || layer_hi > c.n_layers || layer_lo > layer_hi) return CAKE_ERR_ARG;
+  if ((group != 32 && group != 64 && group != 128) || group > c.head_dim) return CAKE_ERR_ARG;
+  if (!row_offsets_out || !kgroup_offsets_out) return CAKE_ERR_ARG;
+  if (layer_hi > ctx->n_evicted || ctx->n_evicted < 1) return CAKE_ERR_STATE;
+  if (ctx->last_alloc != ctx->n_evicted - 1) return CAKE_ERR_STATE;
+  LayerPtrs ptrs;
+  memset(&ptrs, 0, sizeof(ptrs));
+  if (ctx->n_req > 0 && layer_hi > layer_lo) {
+    if (!k_layers || !v_layers || !k_codes || !k_scale || !k_zero || !v_codes || !v_scale || !v_zero)
+      return CAKE_ERR_ARG;
+    for (int l = layer_lo; l < layer_hi; ++l) {
+      if (!k_layers[l] || !v_layers[l]) return CAKE_ERR_ARG;
+      ptrs.k[l] = k_layers[l];
+      ptrs.v[l] = v_layers[l];
+    }
+  }
+  CAKE_CUDA_TRY(main_after_side(ctx, (cudaStream_t)stream));
+  const int sp = prof_begin(ctx, CAKE_PROF_COMPACT, (cudaStream_t)stream);
+  const int32_t rc = launch_compact_int4(ctx, layer_lo, layer_hi, ptrs, group, k_codes, k_scale, k_zero, v_codes,
+                                         v_scale, v_zero, row_offsets_out, kgroup_offsets_out, positions_out,
+                                         (cudaStream_t)stream);
+  prof_end(ctx, sp, (cudaStream_t)stream);
+  return rc;
+}
+
 int64_t cake_packed_rows_bound(const cake_ctx* ctx) {
   if (!ctx) return CAKE_ERR_ARG;
   if (ctx->n_req < 0) return CAKE_ERR_STATE;

@@ -211,6 +211,11 @@ int32_t launch_decode_step(cake_ctx* ctx, int32_t layer, const void* q_new, cons
                            const void* v_new, void* k_cache, void* v_cache, cudaStream_t st);
 int32_t launch_decode_read(cake_ctx* ctx, int32_t req, int32_t layer, int32_t* positions, float* scores,
                            int32_t* slots, cudaStream_t st);
+// quant.cu
+int32_t launch_compact_int4(cake_ctx* ctx, int32_t lo, int32_t hi, const LayerPtrs& ptrs, int32_t group,
+                            uint8_t* k_codes, float* k_scale, float* k_zero, uint8_t* v_codes,
+                            float* v_scale, float* v_zero, int64_t* row_offsets, int64_t* kgroup_offsets,
+                            int32_t* positions, cudaStream_t st);
 // compact.cu
 int32_t launch_compact(cake_ctx* ctx, int32_t lo, int32_t hi, const LayerPtrs& ptrs, void* k_out,
                        void* v_out, int64_t* row_offsets, int32_t* positions, cudaStream_t st);

@@ -205,6 +205,18 @@ int32_t launch_compact(cake_ctx* ctx, int32_t lo, int32_t hi, const LayerPtrs& p
   return cuda_status(cudaGetLastError());
 }
 
+// Packed row offsets and positions of layers [lo, hi): the first half of a compaction.
+int32_t run_packed_positions(cake_ctx* ctx, int32_t lo, int32_t hi, int64_t* row_offsets, int32_t* positions,
+                             cudaStream_t st) {
+  const cake_config& c = ctx->cfg;
+  const int32_t* budget = ctx->d_budget[(ctx->n_evicted - 1) & 1];
+  packed_offsets<<<1, 32, 0, st>>>(budget, row_offsets, ctx->n_req, c.n_layers, lo, hi, c.n_kv_heads,
+                                   c.window);
+  count_launch();
+  if (ctx->n_req == 0 || hi <= lo) return cuda_status(cudaGetLastError());
+  return run_sorted_positions(ctx, 0, ctx->n_req, lo, hi, row_offsets, positions, 0, st);
+}
+
 // Packed row offsets and positions of every layer into context scratch (decode-time set-up).
 int32_t run_sorted_positions_packed(cake_ctx* ctx, const int64_t* offsets_c, int32_t* out, cudaStream_t st) {
   const cake_config& c = ctx->cfg;

@@ -683,3 +683,48 @@ def test_cumulative_attention_brute_force():
                 want[h // 2, j] += e[j] / sum(e) / 2
     assert np.allclose(got, want, rtol=1e-12)
     assert np.allclose(got.sum(axis=1), N)          # every query row sums to one
+
+
+# ------------------------------------------------------- quantised compaction
+def test_int4_codes_properties_and_brute_force():
+    rng = np.random.default_rng(51)
+    x = rng.normal(size=(5, 32)).astype(np.float32)
+    q, s, z = O.int4_codes(x, axis=1)
+    assert q.dtype == np.uint8 and q.min() == 0 and q.max() == 15
+    assert np.array_equal(z[:, 0], x.min(axis=1))
+    for r in range(5):
+        lo, hi = np.float32(x[r].min()), np.float32(x[r].max())
+        sc = np.float32(np.float32(hi - lo) / np.float32(15))
+        assert s[r, 0] == sc
+        for c in range(32):
+            want = int(np.clip(np.rint(np.float32(np.float32(x[r, c] - lo) / sc)), 0, 15))
+            assert q[r, c] == want
+        assert q[r, np.argmin(x[r])] == 0 and q[r, np.argmax(x[r])] == 15
+    deq = z + q.astype(np.float32) * s
+    assert np.all(np.abs(deq - x) <= 0.5 * s * (1 + 1e-5))            # half a step at most
+    # a constant group: scale 1, codes 0, exact reconstruction
+    q, s, z = O.int4_codes(np.full((2, 8), 3.25, dtype=np.float32), axis=1)
+    assert np.all(q == 0) and np.all(s == 1) and np.all(z == 3.25)
+    # ties round to even: (x - zero)/scale = 0.5 -> 0, 1.5 -> 2
+    q, s, z = O.int4_codes(np.array([[0.0, 0.5, 1.5, 15.0]], dtype=np.float32), axis=1)
+    assert list(q[0]) == [0, 0, 2, 15]
+
+
+def test_key_and_value_group_shapes_and_packing():
+    rng = np.random.default_rng(52)
+    v = rng.normal(size=(7, 64)).astype(np.float32)
+    q, s, z = O.quantize_values_per_token(v, 32)
+    assert q.shape == (7, 64) and s.shape == (7, 2) and z.shape == (7, 2)
+    for r in range(7):
+        for gi in range(2):
+            qq, ss, zz = O.int4_codes(v[r, 32 * gi:32 * gi + 32][None], axis=1)
+            assert np.array_equal(q[r, 32 * gi:32 * gi + 32], qq[0]) and s[r, gi] == ss[0, 0]
+    k = rng.normal(size=(70, 64)).astype(np.float32)
+    q, s, z = O.quantize_keys_per_channel(k, 32)
+    assert q.shape == (70, 64) and s.shape == (3, 64)                 # 32 + 32 + 6 rows
+    for c in range(64):
+        qq, ss, zz = O.int4_codes(k[64:70, c][None], axis=1)
+        assert np.array_equal(q[64:70, c], qq[0]) and s[2, c] == ss[0, 0] and z[2, c] == zz[0, 0]
+    packed = O.pack_nibbles(q)
+    assert packed.shape == (70, 32)
+    assert np.array_equal(packed & 15, q[:, 0::2]) and np.array_equal(packed >> 4, q[:, 1::2])
