@@ -81,7 +81,7 @@ struct TcParams {
   long long spin_limit;         // cycles after which a wait gives up and raises CAKE_ERR_TIMEOUT
   int n_pairs;
   int Hkv, Hq, Sw, rows, d;
-  float scale2, gamma, bessel;
+  float scale2, inv_scale2, gamma, bessel;
   int ind_mode;                 // CAKE_IND_*
   int merge_ways;               // rows the merger warp merges side by side: 1, or 2 or 4 when pairs are short
 };
@@ -186,6 +186,28 @@ __device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint32
       ::"r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(idesc), "n"(kAcc), "r"(kDescHi)
       : "memory");
 }
+// The same with an explicit high descriptor word: operands that are not in the 128-byte swizzle.
+template <int kAcc>
+__device__ __forceinline__ void umma_ss_hi(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                           uint32_t hi) {
+  asm volatile(
+      "{\n.reg .pred p, e;\n.reg .b64 da, db;\nsetp.ne.b32 p, %4, 0;\nelect.sync _|e, 0xffffffff;\n"
+      "mov.b64 da, {%1, %5};\nmov.b64 db, {%2, %5};\n"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n}"
+      ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "n"(kAcc), "r"(hi)
+      : "memory");
+}
+// Pass B folds the rows' log-sum-exps into the contraction: one more K = 16 step whose key-side
+// operand holds 1 in its first three columns and whose row-side operand holds -lse / scale split
+// into three bf16 terms, so the accumulator is (q.k - lse/scale) and the statistics warps neither
+// load nor subtract anything per logit.  These two operands are 128 rows x 16 bf16 in the
+// K-major layout without swizzle: 8-row x 16-byte core matrices, the two core matrices of a row
+// group 128 bytes apart (leading-dimension offset), row groups 256 bytes apart (stride offset).
+constexpr uint32_t kExtBytes = 128 * 32;
+constexpr uint32_t kExtDescHi = (256u >> 4) | (1u << 14);            // SBO, version 1, no swizzle
+constexpr uint32_t kExtDescLoLbo = (128u >> 4) << 16;                // LBO field of the low word
+__device__ __forceinline__ uint32_t ext_row_offset(int r) { return (uint32_t)((r >> 3) * 256 + (r & 7) * 16); }
+
 // Copies 128 rows x 32 bytes (one K = 16 slice of a K-major operand) from shared to tensor memory.
 __device__ __forceinline__ void tmem_cp_128x256b(uint32_t tmem_dst, uint64_t sdesc) {
   asm volatile("{\n.reg .pred e;\nelect.sync _|e, 0xffffffff;\n@e tcgen05.cp.cta_group::1.128x256b [%0], %1;\n}"
@@ -234,6 +256,11 @@ __device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
 __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
   f32x2 d;
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
 __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
@@ -287,14 +314,15 @@ struct Smem {
   uint64_t* lse_free;  // [2]
   uint32_t* tmem_holder;
   uint32_t* a_done;    // [NSTATW] pass-A ops whose partial rows each statistics warp has written
-  float* lse;          // [2][128] denominators of the pairs of the current / next pass-B op
+  uint8_t* ext_a;      // the constant key-side operand of the extra K step of pass B
+  uint8_t* ext_b;      // [2] its row-side operand: -lse/scale of the current / next pass-B op
   ScoreOp* ops;        // [kSmemOps] the first ops of this CTA's program
 };
 
 constexpr size_t kQBytes = 2 * SLAB_BYTES;
 constexpr int kSmemOps = 128;        // ops of a CTA's program kept in shared memory
 constexpr size_t kSmemBytes = 1024 /*align*/ + 2 * kQBytes + (size_t)STAGES * 2 * SLAB_BYTES + 320 +
-                              2 * 128 * 4 + kSmemOps * sizeof(ScoreOp) + 64;
+                              128 + 3 * kExtBytes + kSmemOps * sizeof(ScoreOp) + 64;
 
 __device__ __forceinline__ Smem carve(uint8_t* base) {
   Smem s;
@@ -312,7 +340,9 @@ __device__ __forceinline__ Smem carve(uint8_t* base) {
   s.tmem_holder = (uint32_t*)p; p += 8;
   s.a_done = (uint32_t*)p;    p += 4 * 16;
   p = (uint8_t*)(((uintptr_t)p + 15) & ~(uintptr_t)15);
-  s.lse = (float*)p;          p += 2 * 128 * 4;
+  p = (uint8_t*)(((uintptr_t)p + 127) & ~(uintptr_t)127);
+  s.ext_a = p;                p += kExtBytes;
+  s.ext_b = p;                p += 2 * kExtBytes;
   s.ops = (ScoreOp*)p;
   return s;
 }
@@ -349,7 +379,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     for (int i = 0; i < STAGES; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], 1); }
     for (int i = 0; i < NBUF; ++i) { mbar_init(&S.acc_full[i], 1); mbar_init(&S.acc_empty[i], 4); }
     for (int i = 0; i < 2; ++i) { mbar_init(&S.q_full[i], 1); mbar_init(&S.q_empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&S.lse_full[i], 1); mbar_init(&S.lse_free[i], NSTATW); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&S.lse_full[i], 1); mbar_init(&S.lse_free[i], 1); }
     for (int i = 0; i < NSTATW; ++i) S.a_done[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -361,6 +391,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   // rows of the query tiles that TMA never writes must read as zero
   for (int i = threadIdx.x; i < (int)(2 * kQBytes / 16); i += TC_THREADS)
     reinterpret_cast<uint4*>(S.q)[i] = make_uint4(0, 0, 0, 0);
+  // operands of the extra K step: zero, then ones in the first three columns of the key side
+  for (int i = threadIdx.x; i < (int)(3 * kExtBytes / 16); i += TC_THREADS)
+    reinterpret_cast<uint4*>(S.ext_a)[i] = make_uint4(0, 0, 0, 0);
+  __syncthreads();
+  if (threadIdx.x < 128)
+    *reinterpret_cast<uint2*>(S.ext_a + ext_row_offset(threadIdx.x)) = make_uint2(0x3F803F80u, 0x00003F80u);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (warp == WARP_MMA) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -422,13 +458,16 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   } else if (warp == WARP_MMA) {
     // ------------------------------------------------ MMA issuer (converged warp, elected lane issues)
     {
-      uint32_t t = 0, qn = 0;
+      uint32_t t = 0, qn = 0, kbm = 0;
       const uint32_t k_lo0 = (smem_u32(S.k) & 0x3FFFFu) >> 4;
+      const uint32_t ext_a_lo = ((smem_u32(S.ext_a) & 0x3FFFFu) >> 4) | kExtDescLoLbo;
       bool ok = true;
       for (int oi = op_lo; oi < op_hi && ok; ++oi) {
         const ScoreOp op = get_op(oi);
         if (op.nkeys <= 0) continue;
         const uint32_t idesc = op.phase ? instr_desc(128, rows_pad) : instr_desc(128, TILE);
+        const int eslot = kbm & 1;
+        const uint32_t ext_b_lo = ((smem_u32(S.ext_b + eslot * kExtBytes) & 0x3FFFFu) >> 4) | kExtDescLoLbo;
         const int qb = qn & 1;
         ok = mbar_wait(&S.q_full[qb], (qn >> 1) & 1, P.status, P.spin_limit);
         ++qn;
@@ -446,6 +485,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             for (int ks = 0; ks < 4; ++ks)
               tmem_cp_128x256b(tmem_q + (uint32_t)((sl * 4 + ks) * 8),
                                smem_desc(qaddr + sl * SLAB_BYTES + ks * 32));
+        }
+        if (op.phase) {
+          // the rows' -lse/scale operand of this op (written by the denominator warp)
+          ok = mbar_wait(&S.lse_full[eslot], (kbm >> 1) & 1, P.status, P.spin_limit);
+          if (!ok) break;
         }
         const int ntiles = (op.nkeys + TILE - 1) / TILE;
         for (int it = 0; it < ntiles; ++it, ++t) {
@@ -470,6 +514,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
               umma_ss<1>(tmem_d, k_lo + o + 4, q_lo + o + 4, idesc);
               umma_ss<1>(tmem_d, k_lo + o + 6, q_lo + o + 6, idesc);
             }
+            umma_ss_hi<1>(tmem_d, ext_a_lo, ext_b_lo, idesc, kExtDescHi);      // ... - lse/scale
           } else {
             // D[row][key] = Q K^T, queries from tensor memory
             umma_ts<0>(tmem_d, tmem_q, k_lo, idesc);
@@ -488,6 +533,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           umma_commit(&S.acc_full[b]);
         }
         umma_commit(&S.q_empty[qb]);     // query buffer free once every MMA of the op has run
+        if (op.phase) {
+          umma_commit(&S.lse_free[eslot]);   // and so is the op's -lse/scale operand
+          ++kbm;
+        }
       }
     }
   } else if (warp == WARP_MERGE) {
@@ -672,8 +721,24 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       } else {
         v = __ldcg(reinterpret_cast<const float4*>(P.lse2 + (size_t)pair * 128) + lane);
       }
-      // stored negated: the statistics warps add them
-      reinterpret_cast<float4*>(S.lse + slot * 128)[lane] = make_float4(-v.x, -v.y, -v.z, -v.w);
+      // -lse / scale as three bf16 terms (24 bits) in columns 0..2 of the rows' operand
+      {
+        const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int r = 4 * lane + e;
+          const float t = -vv[e] * P.inv_scale2;
+          const __nv_bfloat16 hi = __float2bfloat16_rn(t);
+          const float r1 = t - __bfloat162float(hi);
+          const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+          const uint32_t w0 = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16);
+          const uint32_t w1 = (uint32_t)__bfloat16_as_ushort(lo);
+          *reinterpret_cast<uint2*>(S.ext_b + slot * kExtBytes + ext_row_offset(r)) =
+              r < P.rows ? make_uint2(w0, w1) : make_uint2(0u, 0u);
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&S.lse_full[slot]);
       ++kb;
@@ -693,7 +758,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const int b = wg;
     (void)b;
     uint32_t tmod = 0;                              // tiles of the ops so far, modulo NWG
-    uint32_t fpar = 0, kb = 0;                      // phase parity of my_full; pass-B ops so far
+    uint32_t fpar = 0;                              // phase parity of my_full
     uint32_t n_a_done = 0;                          // pass-A ops this warp has delivered
     bool ok = true;
     for (int oi = op_lo; oi < op_hi; ++oi) {
@@ -704,10 +769,6 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       tmod = (tmod + (uint32_t)ntiles) % NWG;
       if (op.phase) {
         // ---------------- pass B: thread = key, columns = rows r' = i*G + h
-        const int slot = kb & 1;
-        if (ok) ok = mbar_wait(&S.lse_full[slot], (kb >> 1) & 1, P.status, P.spin_limit);
-        ++kb;
-        const float* lse_s = S.lse + slot * 128;
         float vacc[G], hs[G];
 #pragma unroll
         for (int h = 0; h < G; ++h) { vacc[h] = 0.f; hs[h] = 0.f; }
@@ -732,13 +793,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
               __syncwarp();
               if (lane == 0) mbar_arrive(my_empty);
             }
-            // 32 columns = 32/G window rows x G heads; ls = minus the rows' log-sum-exps
-            float ls[32];
-#pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4) {
-              const float4 l4 = reinterpret_cast<const float4*>(lse_s + c0)[q4];
-              ls[q4 * 4 + 0] = l4.x; ls[q4 * 4 + 1] = l4.y; ls[q4 * 4 + 2] = l4.z; ls[q4 * 4 + 3] = l4.w;
-            }
+            // 32 columns = 32/G window rows x G heads; the accumulator is q.k - lse/scale
             if constexpr (G % 2 == 0) {
               // two heads per instruction
               const f32x2 sc2 = pack2(P.scale2, P.scale2);
@@ -748,8 +803,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 #pragma unroll
                 for (int hp = 0; hp < G / 2; ++hp) {
                   const int c = ii * G + 2 * hp;
-                  const f32x2 tt2 = fma2(pack2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), sc2,
-                                         pack2(ls[c], ls[c + 1]));
+                  const f32x2 tt2 = mul2(pack2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), sc2);
                   float t0, t1;
                   unpack2(tt2, t0, t1);
                   const f32x2 p2 = pack2(ex2(t0), ex2(t1));
@@ -769,7 +823,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 float a = 0.f;
 #pragma unroll
                 for (int h = 0; h < G; ++h) {
-                  const float tt = fmaf(__uint_as_float(r[ii * G + h]), P.scale2, ls[ii * G + h]);
+                  const float tt = __uint_as_float(r[ii * G + h]) * P.scale2;
                   const float p = ex2(tt);
                   s1[h] += p;
                   s2[h] = fmaf(p, p, s2[h]);
@@ -803,8 +857,6 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             P.raw[op.base + j] = combine_indicator(P.ind_mode, P.gamma, mean, var, (float)P.Sw);
           }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&S.lse_free[slot]);          // done with this op's denominators
         // fixed-order reduction over the warp's keys
 #pragma unroll
         for (int h = 0; h < G; ++h) {
@@ -1244,6 +1296,7 @@ int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const v
   P.T = ctx->total_tokens;
   P.Hkv = c.n_kv_heads; P.Hq = c.n_q_heads; P.Sw = c.window; P.rows = ctx->rows; P.d = c.head_dim;
   P.scale2 = kLog2e / sqrtf((float)c.head_dim);
+  P.inv_scale2 = 1.f / P.scale2;
   P.gamma = c.gamma;
   P.ind_mode = c.indicator_mode;
   P.merge_ways = ctx->tc_merge_ways;
