@@ -136,6 +136,17 @@ __device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* m
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "l"(policy)
       : "memory");
 }
+// 3-D tiled TMA load with an L2 eviction-priority hint: a whole key tile (both 64-element slabs)
+// in one copy.
+__device__ __forceinline__ void tma_load_3d_hint(void* dst, const CUtensorMap* map, uint64_t* bar,
+                                                 int c0, int c1, int c2, uint64_t policy) {
+  asm volatile(
+      "{\n.reg .pred e;\nelect.sync _|e, 0xffffffff;\n"
+      "@e cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5}], [%2], %6;\n}"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "l"(policy)
+      : "memory");
+}
 __device__ __forceinline__ uint64_t l2_policy_evict_last() {
   uint64_t p;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
@@ -443,9 +454,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           if (!ok) break;
           mbar_expect_tx(&S.full[s], stage_bytes);
           uint8_t* dst = S.k + (size_t)s * 2 * SLAB_BYTES;
-          for (int sl = 0; sl < n_slab; ++sl)
-            tma_load_2d_hint(dst + sl * SLAB_BYTES, &k_map, &S.full[s], sl * 64,
-                             (int)(row0 + it * TILE), pol);
+          // the map's dimensions are (64 elements, key rows, slabs): the box lands slab by slab
+          tma_load_3d_hint(dst, &k_map, &S.full[s], 0, (int)(row0 + it * TILE), 0, pol);
         }
       }
       // do not leave the CTA while a bulk copy may still be writing its shared memory
@@ -1257,11 +1267,13 @@ int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const v
   const int G = c.n_q_heads / c.n_kv_heads;
   CUtensorMap qmap, kmap;
   {
-    const cuuint64_t dims[2] = {(cuuint64_t)c.head_dim, (cuuint64_t)c.n_kv_heads * ctx->total_tokens};
-    const cuuint64_t strides[1] = {(cuuint64_t)c.head_dim * 2};
-    const cuuint32_t box[2] = {64, TILE};
-    const cuuint32_t es[2] = {1, 1};
-    if (enc(&kmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(k), dims, strides, box, es,
+    // K [rows][d] seen as (64 elements, rows, d/64 slabs): one box of 128 rows brings both
+    // 64-element halves of the rows, each as its own 128-byte-swizzled slab
+    const cuuint64_t dims[3] = {64, (cuuint64_t)c.n_kv_heads * ctx->total_tokens, (cuuint64_t)(c.head_dim / 64)};
+    const cuuint64_t strides[2] = {(cuuint64_t)c.head_dim * 2, 128};
+    const cuuint32_t box[3] = {64, TILE, (cuuint32_t)(c.head_dim / 64)};
+    const cuuint32_t es[3] = {1, 1, 1};
+    if (enc(&kmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(k), dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return CAKE_ERR_CUDA;
