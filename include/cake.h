@@ -240,7 +240,9 @@ int32_t cake_status(cake_ctx* ctx, int32_t* device_status_out, void* stream);
 #define CAKE_PROF_COMPACT     4
 #define CAKE_PROF_KINDS       5
 /* While enabled, every stage of the path brackets its kernels with CUDA events
- * on the caller's stream (this perturbs back-to-back launches slightly). */
+ * on the stream the stage runs on: the caller's stream for the score kernel and
+ * the compaction, the context's own streams for pooling/preference, budgets and
+ * eviction (this perturbs back-to-back launches slightly). */
 int32_t cake_profile_enable(cake_ctx* ctx, int32_t on);
 /* Synchronises `stream`; returns, per CAKE_PROF_* kind, the milliseconds and
  * the number of bracketed spans accumulated since the last read (HOST arrays

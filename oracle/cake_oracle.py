@@ -36,9 +36,10 @@ parameter so the alternative can be exercised):
 Pins: tests/test_oracle_pins.py checks every function below against closed
 forms, invariants the paper states (Proposition 1, Theorem 2), special cases
 (gamma = 0, kernel 1, single layer) and brute force on tiny inputs.  What no
-pin can decide from the paper's text -- max versus average pooling, ddof, and
-whether the budget counts the window -- is "parity unpinned" beyond those
-readings.
+pin can decide from the paper's text -- max versus average pooling, ddof,
+whether the budget counts the window, how the decode step's "update_score"
+combines old and new values, and the rounding rule of the 4-bit compaction --
+is "parity unpinned" beyond those readings.
 """
 from __future__ import annotations
 

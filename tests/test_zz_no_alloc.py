@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import cake_oracle as O
 from paper_2503_12491_b200 import binding
 from paper_2503_12491_b200.binding import Cake, CakeError, CAKE_ERR_ARG, CAKE_ERR_CAPACITY
 
@@ -55,11 +56,10 @@ def test_static_selection_matches_context_path_twice_in_a_row():
         torch.cuda.synchronize()
         assert torch.equal(out, want), f"call {call}"
         assert torch.equal(out[0].cpu(), torch.arange(keep, dtype=torch.int32))
-        # and against a plain definition: value descending, position ascending
+        # and against the oracle's TopK of Eq. 12: value descending, position ascending
         v = vals.cpu().numpy().astype(np.float64)
         for h in range(heads):
-            order = np.lexsort((np.arange(n), -v[h]))
-            assert np.array_equal(out[h].cpu().numpy(), np.sort(order[:keep]))
+            assert np.array_equal(out[h].cpu().numpy(), O.topk_keep(v[h], keep))
 
 
 def test_static_selection_rejects_what_does_not_fit():
