@@ -126,16 +126,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_
   }
   return true;
 }
-// 2-D tiled TMA load with an L2 eviction-priority hint (a policy made by createpolicy).
-__device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* map, uint64_t* bar,
-                                                 int c0, int c1, uint64_t policy) {
-  asm volatile(
-      "{\n.reg .pred e;\nelect.sync _|e, 0xffffffff;\n"
-      "@e cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-      "[%0], [%1, {%3, %4}], [%2], %5;\n}"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "l"(policy)
-      : "memory");
-}
 // 3-D tiled TMA load with an L2 eviction-priority hint: a whole key tile (both 64-element slabs)
 // in one copy.
 __device__ __forceinline__ void tma_load_3d_hint(void* dst, const CUtensorMap* map, uint64_t* bar,
@@ -650,22 +640,23 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             while (ld_acquire(&P.pair_cnt[pair]) < want) {
               publish();
               if (clock64() - t0 > P.spin_limit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
-              __nanosleep(100);
+              __nanosleep(40);
             }
             if (!ok) break;
             waited = true;
           }
           float4 acc = make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
-          for (int base = s_lo; base < s_hi; base += 32 * 8) {
-            float4 pv[8];
+          // 12 loads per lane in flight: the 384 partials of a row at 128 CTAs come in one round trip
+          for (int base = s_lo; base < s_hi; base += 32 * 12) {
+            float4 pv[12];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 12; ++u) {
               const int sg = base + u * 32 + lane;
               pv[u] = sg < s_hi ? __ldcg(&P.rowpart[(size_t)sg * 128 + r])
                                 : make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) acc = merge_rows(acc, pv[u]);
+            for (int u = 0; u < 12; ++u) acc = merge_rows(acc, pv[u]);
           }
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) {
@@ -712,7 +703,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           const long long t0 = clock64();
           while (ld_acquire(&P.pair_done[pair]) < want) {
             if (clock64() - t0 > P.spin_limit) { atomicCAS(P.status, 0, CAKE_ERR_TIMEOUT); ok = false; break; }
-            __nanosleep(64);
+            __nanosleep(32);
           }
         }
       }
