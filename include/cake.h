@@ -320,6 +320,18 @@ int32_t cake_debug_skew_sync(cake_ctx* ctx, int32_t delta);
  * CTAs' programs, [7] SMs left to the cascade kernels.  Entries [1]..[6] are 0 on the SIMT path. */
 int32_t cake_plan_info(const cake_ctx* ctx, int32_t* out8);
 
+/* Builds the score kernel's launch plan for a batch on the HOST alone (no device, no context: it
+ * runs without a GPU) and checks what the kernel relies on: every key tile covered exactly once
+ * per pass, every CTA's program ordered so that a wave's column pass can only wait for row-pass
+ * ops that wait for nothing, merge groups within two adjacent waves, table sizes.  n_sm = SMs of
+ * the device to plan for, reserved_sms as CAKE_RESERVED_SMS.  info8 (HOST, 8 int32): CTAs,
+ * waves, merge ways, pass-A segments, pass-B segments, ops of the two-pass programs, ops of the
+ * column-pass-only programs, and the number of the violated property (0 = none).  Returns
+ * CAKE_OK, CAKE_ERR_ARG (also when the shape takes the SIMT path), an error of the plan builder,
+ * or CAKE_ERR_STATE when a property is violated. */
+int32_t cake_plan_check(const cake_config* cfg, int32_t n_sm, int32_t reserved_sms, int32_t n_req,
+                        const int64_t* cu_seqlens_host, int32_t* info8);
+
 /* ---- selection without any allocation ------------------------------------- */
 /* The paper has no counterpart for this entry point; it exists for callers that are not
  * allowed to allocate device memory when they call in: code running inside another

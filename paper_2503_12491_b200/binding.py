@@ -31,7 +31,7 @@ EXPORTS = [
     "cake_profile_enable", "cake_profile_read", "cake_uses_tensor_cores",
     "cake_select_positions_static", "cake_plan_info", "cake_set_wait_limit", "cake_debug_skew_sync",
     "cake_decode_rows_bound", "cake_decode_begin", "cake_decode_step", "cake_decode_get_state",
-    "cake_compact_int4",
+    "cake_compact_int4", "cake_plan_check",
 ]
 PROF_KINDS = ["score", "finalize", "allocate", "evict", "compact"]
 
@@ -92,6 +92,8 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.cake_uses_tensor_cores.argtypes = [vp]
     lib.cake_select_positions_static.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.cake_plan_info.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.cake_plan_check.argtypes = [ctypes.POINTER(CakeConfig), i32, i32, i32, ctypes.POINTER(i64),
+                                    ctypes.POINTER(i32)]
     lib.cake_decode_rows_bound.argtypes = [vp]
     lib.cake_decode_rows_bound.restype = i64
     lib.cake_decode_begin.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, vp, vp, i32, vp]

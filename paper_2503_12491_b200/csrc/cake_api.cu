@@ -720,6 +720,15 @@ int32_t cake_debug_skew_sync(cake_ctx* ctx, int32_t delta) {
   return CAKE_OK;
 }
 
+int32_t cake_plan_check(const cake_config* cfg, int32_t n_sm, int32_t reserved_sms, int32_t n_req,
+                        const int64_t* cu_seqlens_host, int32_t* info8) {
+  if (!cfg || !info8 || n_sm < 1 || reserved_sms < 0 || n_req < 0 || (n_req > 0 && !cu_seqlens_host))
+    return CAKE_ERR_ARG;
+  for (int r = 0; r < n_req; ++r)
+    if (cu_seqlens_host[r + 1] - cu_seqlens_host[r] < cfg->window) return CAKE_ERR_ARG;
+  return tc_plan_check(*cfg, n_sm, reserved_sms, n_req, cu_seqlens_host, info8);
+}
+
 int32_t cake_plan_info(const cake_ctx* ctx, int32_t* out8) {
   if (!ctx || !out8) return CAKE_ERR_ARG;
   if (ctx->n_req < 0) return CAKE_ERR_STATE;

@@ -198,6 +198,8 @@ int32_t launch_score_simt(cake_ctx* ctx, int32_t layer, const void* q_win, const
 bool tc_path_supported(const cake_config& c);
 int64_t tc_max_segments(const cake_config& c, int n_sm);
 int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req);
+int32_t tc_plan_check(const cake_config& c, int n_sm, int reserved, int32_t n_req, const int64_t* cu,
+                      int32_t* info8);
 int32_t launch_score_tc(cake_ctx* ctx, int32_t layer, const void* q_win, const void* k,
                         const float* lse, cudaStream_t st);
 // cascade.cu

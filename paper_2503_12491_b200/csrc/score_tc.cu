@@ -38,6 +38,7 @@
 #include <math_constants.h>
 
 #include <algorithm>
+#include <cstring>
 #include <vector>
 
 namespace cake {
@@ -1244,6 +1245,107 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
     };
     while (ways > 1 && !span_ok(ways)) ways >>= 1;
     ctx->tc_merge_ways = ways;
+  }
+  return CAKE_OK;
+}
+
+// Builds the plan of a batch on the host alone (no device, no context) and checks the properties
+// the kernel relies on.  Returns CAKE_OK, an error of the plan builder, or CAKE_ERR_STATE with
+// info8[7] = the number of the violated property:
+//   1  every key tile of every pair is covered exactly once by the pass-A ops, and every non-window
+//      tile exactly once by the pass-B ops
+//   2  inside every CTA's program the pass-B ops come in non-decreasing wave order and every
+//      pass-A op of a wave w' <= w precedes the first pass-B op of wave w (so a wave's pass B can
+//      only ever wait for pass-A ops that wait for nothing themselves)
+//   3  the pairs the merger warps handle side by side lie in at most two adjacent waves
+//   4  op counts and segment numbers stay inside the tables the context would allocate
+int32_t tc_plan_check(const cake_config& c, int n_sm, int reserved, int32_t n_req, const int64_t* cu,
+                      int32_t* info8) {
+  if (!tc_path_supported(c)) return CAKE_ERR_ARG;
+  cake_ctx x;
+  memset(&x, 0, sizeof(x));
+  x.cfg = c;
+  x.n_sm = n_sm;
+  x.n_sm_score = n_sm - reserved > 0 ? n_sm - reserved : 1;
+  const int Hkv = c.n_kv_heads, n_pairs = n_req * Hkv;
+  std::vector<ReqInfo> reqs(n_req > 0 ? n_req : 1);
+  for (int r = 0; r < n_req; ++r) {
+    memset(&reqs[r], 0, sizeof(ReqInfo));
+    reqs[r].cu = cu[r];
+    reqs[r].N = (int32_t)(cu[r + 1] - cu[r]);
+    reqs[r].n = reqs[r].N - c.window;
+  }
+  x.h_req = reqs.data();
+  x.max_tc_segs = (int32_t)tc_max_segments(c, n_sm);
+  x.max_tc_ops = 3 * x.max_tc_segs + 8;
+  std::vector<ScoreOp> ops((size_t)x.max_tc_ops);
+  std::vector<int32_t> index(2 * (size_t)(n_pairs + 1) + 2 * (size_t)(n_sm + 1));
+  x.h_tc_ops = ops.data();
+  x.h_tc_index = index.data();
+  const int32_t rc = tc_build_plan(&x, n_req);
+  info8[0] = x.n_tc_ctas; info8[1] = x.n_tc_waves; info8[2] = x.tc_merge_ways; info8[3] = x.n_tc_asegs;
+  info8[4] = x.n_tc_bsegs; info8[5] = x.n_tc_ops_full; info8[6] = x.n_tc_ops_b; info8[7] = 0;
+  if (rc != CAKE_OK || x.n_tc_ctas == 0) return rc;
+  auto fail = [&](int what) { info8[7] = what; return (int32_t)CAKE_ERR_STATE; };
+  if (x.n_tc_ops_full + x.n_tc_ops_b > x.max_tc_ops || x.n_tc_asegs > x.max_tc_segs ||
+      x.n_tc_bsegs > x.max_tc_segs) return fail(4);
+  // waves as the builder forms them
+  std::vector<int> wave_of(n_pairs, 0);
+  {
+    int64_t bytes = 0;
+    int wv = 0;
+    for (int p = 0; p < n_pairs; ++p) {
+      const int64_t pb = (int64_t)reqs[p / Hkv].N * c.head_dim * 2;
+      if (bytes > 0 && bytes + pb > kWaveBytes) { ++wv; bytes = 0; }
+      bytes += pb;
+      wave_of[p] = wv;
+    }
+  }
+  const int32_t* cta_full = index.data() + 2 * (n_pairs + 1);
+  // 1: coverage, per pair and pass, in tiles
+  std::vector<std::vector<int>> cover[2];
+  for (int ph = 0; ph < 2; ++ph) {
+    cover[ph].resize(n_pairs);
+    for (int p = 0; p < n_pairs; ++p) {
+      const ReqInfo& rq = reqs[p / Hkv];
+      cover[ph][p].assign(((ph ? rq.n : rq.N) + TILE - 1) / TILE, 0);
+    }
+  }
+  for (int cta = 0; cta < x.n_tc_ctas; ++cta) {
+    int last_b_wave = -1;
+    std::vector<int> first_b_pos(x.n_tc_waves + 1, -1);
+    std::vector<int> last_a_pos(x.n_tc_waves + 1, -1);
+    for (int o = cta_full[cta]; o < cta_full[cta + 1]; ++o) {
+      const ScoreOp& op = ops[o];
+      const int p = op.req * Hkv + op.g;
+      if (p < 0 || p >= n_pairs || op.key0 % TILE != 0 || op.nkeys <= 0) return fail(1);
+      if (op.seg < 0 || op.seg >= (op.phase ? x.n_tc_bsegs : x.n_tc_asegs)) return fail(4);
+      const int t0 = op.key0 / TILE, t1 = (op.key0 + op.nkeys + TILE - 1) / TILE;
+      if (t1 > (int)cover[op.phase][p].size()) return fail(1);
+      for (int t = t0; t < t1; ++t) cover[op.phase][p][t] += 1;
+      const int wv = wave_of[p], pos = o - cta_full[cta];
+      if (op.phase) {
+        if (wv < last_b_wave) return fail(2);
+        last_b_wave = wv;
+        if (first_b_pos[wv] < 0) first_b_pos[wv] = pos;
+      } else {
+        last_a_pos[wv] = pos;
+      }
+    }
+    for (int w = 0; w < x.n_tc_waves; ++w)
+      if (first_b_pos[w] >= 0)
+        for (int w2 = 0; w2 <= w; ++w2)
+          if (last_a_pos[w2] > first_b_pos[w]) return fail(2);
+  }
+  for (int ph = 0; ph < 2; ++ph)
+    for (int p = 0; p < n_pairs; ++p)
+      for (int v : cover[ph][p])
+        if (v != 1) return fail(1);
+  // 3: merge groups
+  const int ways = x.tc_merge_ways;
+  for (int p0 = 0; p0 < n_pairs; p0 += ways) {
+    const int p1 = std::min(n_pairs, p0 + ways) - 1;
+    if (wave_of[p1] - wave_of[p0] > kWaveDepth) return fail(3);
   }
   return CAKE_OK;
 }
