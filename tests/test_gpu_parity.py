@@ -224,7 +224,7 @@ def test_end_to_end_own_indicators_differ_only_near_threshold(case):
                 if diff.size:
                     thr = np.sort(inds[l][g])[::-1][b - 1]
                     rel = np.abs(inds[l][g][diff] - thr) / thr
-                    assert rel.max() <= 2 * RTOL, (r, l, g, diff, rel.max())
+                    assert rel.max() <= RTOL, (r, l, g, diff, rel.max())
     assert cake.status() == 0
     cake.destroy()
 
@@ -310,7 +310,7 @@ def test_one_full_size_layer_of_the_128k_workload():
         if diff.size:
             thr = np.sort(ref["indicator"][g])[::-1][b - 1]
             rel = np.abs(ref["indicator"][g][diff] - thr) / thr
-            assert rel.max() <= 2 * RTOL, (g, diff.size, rel.max())
+            assert rel.max() <= RTOL, (g, diff.size, rel.max())
         if np.isin(needles, want).all():              # the oracle keeps every needle: so must we
             assert np.isin(needles, got[g][:b]).all(), g
         src = ks[0][g, torch.from_numpy(got[g]).long().cuda()]
@@ -358,7 +358,7 @@ def test_four_full_size_layers_through_the_pipelined_cascade():
             if diff.size:
                 thr = np.sort(ref[l]["indicator"][g])[::-1][b - 1]
                 rel = np.abs(ref[l]["indicator"][g][diff] - thr) / thr
-                assert rel.max() <= 2 * RTOL, (l, g, diff.size, rel.max())
+                assert rel.max() <= RTOL, (l, g, diff.size, rel.max())
         g = l % w.n_kv_heads                               # one head's rows per layer, bit for bit
         src = ks[l][g, torch.from_numpy(pb[0][l][g].cpu().numpy()).long().cuda()]
         assert torch.equal(kb[0][l][g], src)
