@@ -316,7 +316,7 @@ int32_t cake_debug_skew_sync(cake_ctx* ctx, int32_t delta);
  * built on the host in cake_begin; nothing here touches the device).  out8 is a HOST array of 8
  * int32: [0] 1 if the tensor-core kernels are used, [1] CTAs of the score kernel, [2] waves (groups
  * of (request, KV head) pairs whose keys pass A and pass B share through L2), [3] rows the merger
- * warps combine side by side (1, 2 or 4), [4] pass-A segments, [5] pass-B segments, [6] ops in the
+ * warps combine side by side (a power of two, 1 to 32), [4] pass-A segments, [5] pass-B segments, [6] ops in the
  * CTAs' programs, [7] SMs left to the cascade kernels.  Entries [1]..[6] are 0 on the SIMT path. */
 int32_t cake_plan_info(const cake_ctx* ctx, int32_t* out8);
 

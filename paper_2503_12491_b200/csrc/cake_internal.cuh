@@ -181,7 +181,7 @@ struct cake_ctx {
   int32_t* h_tc_index;
   int32_t* d_tc_index;
   uint32_t* d_tc_sync;            // [max_pairs] delivered partial rows, then [max_pairs] merged rows
-  int tc_merge_ways;              // rows the merger warp handles side by side (1, 2 or 4), chosen with the plan
+  int tc_merge_ways;              // rows the merger warp handles side by side (a power of two up to 32), chosen with the plan
   float4* d_tc_rowpart;           // [max_tc_segs][kScoreGroups][128]
   float* d_lse2_tc;               // [max_requests][H_kv][128], rows in tile order i*G + h
   float* d_hrow[2];               // [max_pairs][128] sum_j p log2 p per window row, by layer parity

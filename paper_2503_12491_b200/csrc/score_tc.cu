@@ -84,7 +84,7 @@ struct TcParams {
   int Hkv, Hq, Sw, rows, d;
   float scale2, inv_scale2, gamma, bessel;
   int ind_mode;                 // CAKE_IND_*
-  int merge_ways;               // rows the merger warp merges side by side: 1, or 2 or 4 when pairs are short
+  int merge_ways;               // rows the merger warp merges side by side: 1, or 2 to 32 when pairs are short
 };
 
 // ------------------------------------------------------------------ PTX
@@ -569,7 +569,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       };
       if (P.merge_ways > 1) {
         // Short pairs (a ragged batch, MHA): a wave holds several pairs whose rows have few
-        // partials each, so the rows of `ways` (2 or 4) consecutive pairs are merged side by side,
+        // partials each, so the rows of `ways` (2 to 32) consecutive pairs are merged side by side,
         // by 32 / ways lanes each, and the wave's denominators are ready that much sooner.
         const int ways = P.merge_ways, lpr = 32 / ways;         // lanes per row
         const int sub = lane / lpr, l8 = lane % lpr;
@@ -1238,7 +1238,10 @@ int32_t tc_build_plan(cake_ctx* ctx, int32_t n_req) {
     int max_segs = 0;
     for (int p = 0; p < n_pairs; ++p) max_segs = std::max(max_segs, pair_aseg[p + 1] - pair_aseg[p]);
     const int partials = max_segs * NWG;
-    int ways = n_pairs < 4 ? 1 : partials <= 128 ? 4 : partials <= 256 ? 2 : 1;
+    // at most 16 partials per lane (two batches of loads): 32 lanes / ways per row
+    int ways = 1;
+    while (ways < 32 && 2 * ways <= n_pairs && partials * 2 * ways <= 512) ways *= 2;
+    if (n_pairs < 4) ways = 1;
     // The merger handles `ways` consecutive pairs at once and waits for the pass A of all of them.
     // A CTA's program only guarantees A(w+1) before B(w): a group that reached from wave w into
     // wave w+2 would make B(w) wait for an A(w+2) that comes after it.  So every group must lie
