@@ -85,6 +85,9 @@ void free_ctx(cake_ctx* c) {
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   if (c->ev_pool_side) cudaEventDestroy(c->ev_pool_side);
   for (int i = 0; i < 2; ++i) if (c->ev_evict[i]) cudaEventDestroy(c->ev_evict[i]);
+  for (int i = 0; i < 2; ++i) if (c->ev_alloc[i]) cudaEventDestroy(c->ev_alloc[i]);
+  if (c->ev_alloc_main) cudaEventDestroy(c->ev_alloc_main);
+  if (c->alloc_st) cudaStreamDestroy(c->alloc_st);
   if (c->pool_st) cudaStreamDestroy(c->pool_st);
   if (c->side2) cudaStreamDestroy(c->side2);
   if (c->side) cudaStreamDestroy(c->side);
@@ -104,6 +107,7 @@ cudaError_t side_after(cake_ctx* c, cudaStream_t st) {
   cudaError_t e = cudaEventRecord(c->ev_main, st);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_main, 0);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(c->pool_st, c->ev_main, 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(c->alloc_st, c->ev_main, 0);
   return e;
 }
 // Orders the caller's stream after everything enqueued so far on the internal streams.
@@ -112,6 +116,8 @@ cudaError_t main_after_side(cake_ctx* c, cudaStream_t st) {
   if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_side, 0);
   if (e == cudaSuccess) e = cudaEventRecord(c->ev_pool_side, c->pool_st);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_pool_side, 0);
+  if (e == cudaSuccess) e = cudaEventRecord(c->ev_alloc_main, c->alloc_st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_alloc_main, 0);
   return e;
 }
 
@@ -191,6 +197,10 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   ok = ok && cudaStreamCreateWithFlags(&x->side2, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&x->pool_st, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&x->ev_pool_side, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&x->alloc_st, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&x->ev_alloc_main, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; i < 2; ++i)
+    ok = ok && cudaEventCreateWithFlags(&x->ev_alloc[i], cudaEventDisableTiming) == cudaSuccess;
   for (int i = 0; i < 2; ++i)
     ok = ok && cudaEventCreateWithFlags(&x->ev_evict[i], cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&x->ev_fork, cudaEventDisableTiming) == cudaSuccess;
@@ -420,12 +430,18 @@ int32_t cake_allocate(cake_ctx* ctx, int32_t stage, void* stream) {
   if (stage < 0 || stage >= ctx->cfg.n_layers) return CAKE_ERR_ARG;
   if (stage >= ctx->n_pref) return CAKE_ERR_STATE;
   (void)stream;                      // ordered by the internal streams
-  // the newest layer's preference comes from the pooling stream
-  if (ctx->pool_recorded[stage & 1]) CAKE_CUDA_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_pool[stage & 1], 0));
-  const int sp = prof_begin(ctx, CAKE_PROF_ALLOCATE, ctx->side);
-  int32_t rc = launch_allocate(ctx, stage, ctx->side);
-  prof_end(ctx, sp, ctx->side);
+  // The budgets have a stream of their own, so that those of stage m are computed beside the
+  // eviction of stage m-1.  They need the newest layer's preference (pooling stream), and their
+  // buffer was last read by the eviction of stage m-2; the budgets of stage m-1, which they fall
+  // back to, were written on this stream.
+  cudaStream_t ast = ctx->alloc_st;
+  if (ctx->pool_recorded[stage & 1]) CAKE_CUDA_TRY(cudaStreamWaitEvent(ast, ctx->ev_pool[stage & 1], 0));
+  if (ctx->evict_recorded[stage & 1]) CAKE_CUDA_TRY(cudaStreamWaitEvent(ast, ctx->ev_evict[stage & 1], 0));
+  const int sp = prof_begin(ctx, CAKE_PROF_ALLOCATE, ast);
+  int32_t rc = launch_allocate(ctx, stage, ast);
+  prof_end(ctx, sp, ast);
   if (rc != CAKE_OK) return rc;
+  CAKE_CUDA_TRY(cudaEventRecord(ctx->ev_alloc[stage & 1], ast));
   ctx->alloc_of_buf[stage & 1] = stage;
   ctx->last_alloc = stage;
   return CAKE_OK;
@@ -438,6 +454,7 @@ int32_t cake_evict(cake_ctx* ctx, int32_t stage, void* stream) {
   if (ctx->alloc_of_buf[stage & 1] != stage) return CAKE_ERR_STATE;
   if (stage > 0 && ctx->alloc_of_buf[(stage + 1) & 1] != stage - 1) return CAKE_ERR_STATE;
   (void)stream;
+  CAKE_CUDA_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_alloc[stage & 1], 0));
   const int sp = prof_begin(ctx, CAKE_PROF_EVICT, ctx->side);
   int32_t rc = launch_evict(ctx, stage, ctx->side);
   prof_end(ctx, sp, ctx->side);

@@ -95,6 +95,9 @@ struct cake_ctx {
   cudaStream_t side;
   cudaStream_t side2;               // older layers' thresholds of a stage, beside the newest layer's scatter
   cudaStream_t pool_st;             // pooling + preference of layer l+1, beside the budgets and eviction of layer l
+  cudaStream_t alloc_st;            // budgets of stage m, beside the eviction of stage m-1
+  cudaEvent_t ev_alloc[2];          // budgets of a stage of that parity are written
+  cudaEvent_t ev_alloc_main;        // scratch event: budget stream -> caller's
   cudaEvent_t ev_main, ev_side;     // scratch events: caller's stream -> side, side -> caller's
   cudaEvent_t ev_fork, ev_join;     // side -> side2 and back
   cudaEvent_t ev_pool_side;         // scratch event: pooling stream -> caller's
