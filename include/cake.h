@@ -167,7 +167,11 @@ int32_t cake_evict(cake_ctx* ctx, int32_t stage, void* stream);
  * V^ = V[D,:]) into the packed cache.  All of those layers must have been
  * evicted.
  *   k_layers, v_layers  HOST arrays [n_layers] of device pointers, each
- *                       [H_kv][T][d]; entries outside [layer_lo, layer_hi) are ignored
+ *                       [H_kv][T][d]; entries outside [layer_lo, layer_hi) are ignored.
+ *                       A pointer may also be page-locked host memory that the device can
+ *                       address (cudaHostAlloc under unified addressing): the gather then reads
+ *                       only the retained rows over the bus, so values that the scoring never
+ *                       touches need not be copied to the device at all
  *   k_out, v_out        device, capacity >= cake_packed_rows_bound() rows of d elements
  *   row_offsets_out     device int64 [n_req*L + 1]: block (r,l) = index r*L+l occupies
  *                       rows row_offsets[r*L+l] .. row_offsets[r*L+l+1]-1 and is laid

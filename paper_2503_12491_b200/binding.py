@@ -127,11 +127,13 @@ def _check(code: int, where: str) -> None:
         raise CakeError(code, where)
 
 
-def _ptr(t: Optional[torch.Tensor], dtype: Optional[torch.dtype] = None) -> Optional[int]:
+def _ptr(t: Optional[torch.Tensor], dtype: Optional[torch.dtype] = None,
+         pinned_ok: bool = False) -> Optional[int]:
     if t is None:
         return None
-    if not t.is_cuda:
-        raise ValueError("libcake takes CUDA tensors only")
+    if not t.is_cuda and not (pinned_ok and t.is_pinned()):
+        raise ValueError("libcake takes CUDA tensors only" +
+                         (" (or pinned host tensors here)" if pinned_ok else ""))
     if not t.is_contiguous():
         raise ValueError("tensor must be contiguous")
     if dtype is not None and t.dtype != dtype:
@@ -236,8 +238,10 @@ class Cake:
             row_offsets = torch.empty(self.n_req * L + 1, dtype=torch.int64, device=dev)
         if positions is None and want_positions:
             positions = torch.empty(max(rows, 1), dtype=torch.int32, device=dev)
-        kp = (ctypes.c_void_p * L)(*[(_ptr(t, self.dtype) if t is not None else None) for t in k_layers])
-        vp = (ctypes.c_void_p * L)(*[(_ptr(t, self.dtype) if t is not None else None) for t in v_layers])
+        # K/V of a layer may also live in pinned host memory: the gather then fetches only the
+        # retained rows over the bus
+        kp = (ctypes.c_void_p * L)(*[(_ptr(t, self.dtype, True) if t is not None else None) for t in k_layers])
+        vp = (ctypes.c_void_p * L)(*[(_ptr(t, self.dtype, True) if t is not None else None) for t in v_layers])
         _check(self.lib.cake_compact(self._h, layer_lo, hi, kp, vp, _ptr(k_out), _ptr(v_out),
                                      _ptr(row_offsets, torch.int64), _ptr(positions, torch.int32),
                                      _stream()), "cake_compact")

@@ -557,6 +557,25 @@ def test_runs_are_bitwise_reproducible():
     assert torch.equal(outs[0][3], outs[1][3])
 
 
+def test_compaction_reads_values_from_pinned_host_memory():
+    """V (and K) handed to the gather as page-locked host tensors give the same packed cache as
+    device tensors: only the retained rows cross the bus."""
+    w = SMALL_CASES["ragged"]()
+    qs, ks, vs = harness.device_inputs(w)
+    cake = harness.cake_for(w)
+    k_dev, v_dev, off_dev, pos_dev = [t.clone() for t in cake.run(qs, ks, vs, w.cu_seqlens)]
+    hv = [v.cpu().pin_memory() for v in vs]
+    hk = [k.cpu().pin_memory() for k in ks]
+    k_h, v_h, off_h, pos_h = cake.compact(hk, hv)
+    n = int(off_dev[-1])
+    assert n > 0 and torch.equal(off_dev, off_h)
+    assert torch.equal(k_dev[:n], k_h[:n]) and torch.equal(v_dev[:n], v_h[:n])
+    assert torch.equal(pos_dev[:n], pos_h[:n])
+    with pytest.raises(ValueError):
+        cake.compact(ks, [v.cpu() for v in vs])          # pageable host memory is refused
+    cake.destroy()
+
+
 def test_generator_is_bit_identical_on_cpu_and_gpu():
     w = SMALL_CASES["gqa-bf16"]()
     q0, k0, v0 = synth.layer_inputs(w, 1, "cpu")
