@@ -289,7 +289,8 @@ int32_t cake_uses_tensor_cores(const cake_ctx* ctx);
  *                       window entries), slots_out int32 [H_kv][len] (slot of each entry inside
  *                       its head's cap slots); any may be NULL.
  * A head with more than 200 KB / (4 * (G + 1)) slots (10239 at G = 4) does not fit the step
- * kernel's shared memory: cake_decode_begin then returns CAKE_ERR_CAPACITY. */
+ * kernel's shared memory and works in a global-memory area of the context instead (same
+ * results, a slower step for that head). */
 int64_t cake_decode_rows_bound(const cake_ctx* ctx);
 int32_t cake_decode_begin(cake_ctx* ctx, const void* const* k_layers, const void* const* v_layers,
                           void* k_cache, void* v_cache, int64_t* row_offsets_out, int32_t update_mode,

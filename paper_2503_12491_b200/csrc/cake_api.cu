@@ -67,7 +67,7 @@ void free_ctx(cake_ctx* c) {
   cudaFree(c->d_rowpart); cudaFree(c->d_colpart[0]); cudaFree(c->d_colpart[1]);
   cudaFree(c->d_tc_ops); cudaFree(c->d_tc_index); cudaFree(c->d_tc_sync);
   cudaFree(c->d_tc_rowpart); cudaFree(c->d_lse2_tc); cudaFree(c->d_hrow[0]); cudaFree(c->d_hrow[1]);
-  cudaFree(c->d_dec_off); cudaFree(c->d_dec_packed_off); cudaFree(c->d_dec_score); cudaFree(c->d_dec_pos);
+  cudaFree(c->d_dec_off); cudaFree(c->d_dec_packed_off); cudaFree(c->d_dec_score); cudaFree(c->d_dec_tmp); cudaFree(c->d_dec_pos);
   cudaFree(c->d_dec_order); cudaFree(c->d_dec_meta);
   if (c->h_budget_stage) cudaFreeHost(c->h_budget_stage);
   if (c->h_tc_ops) cudaFreeHost(c->h_tc_ops);
@@ -271,6 +271,8 @@ int32_t cake_create(const cake_config* cfg, cake_ctx** out) {
   ok = ok && dev_alloc(&x->d_dec_off, (size_t)R * c.n_layers + 1) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_dec_packed_off, (size_t)R * c.n_layers + 1) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_dec_score, (size_t)x->dec_rows_cap) == cudaSuccess;
+  ok = ok && dev_alloc(&x->d_dec_tmp, (size_t)c.n_kv_heads * (size_t)(c.n_q_heads / c.n_kv_heads + 1) *
+                                          (size_t)(T + R)) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_dec_pos, (size_t)x->dec_rows_cap) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_dec_order, (size_t)x->dec_rows_cap) == cudaSuccess;
   ok = ok && dev_alloc(&x->d_dec_meta, (size_t)x->max_lists) == cudaSuccess;
@@ -686,7 +688,8 @@ int32_t cake_decode_begin(cake_ctx* ctx, const void* const* k_layers, const void
     }
   }
   CAKE_CUDA_TRY(main_after_side(ctx, st));
-  // the step kernel's shared memory is sized from the largest head: read the final budgets back
+  // the step kernel's shared memory is sized from the largest head (up to its limit): read the
+  // final budgets back
   ctx->dec_max_cap = 1;
   if (ctx->n_req > 0) {
     const size_t nb = sizeof(int32_t) * ctx->n_req * c.n_layers;
@@ -697,8 +700,6 @@ int32_t cake_decode_begin(cake_ctx* ctx, const void* const* k_layers, const void
       const int64_t cap = (int64_t)ctx->h_budget_stage[i] + c.window + 1;
       if (cap > ctx->dec_max_cap) ctx->dec_max_cap = cap;
     }
-    const int G = c.n_q_heads / c.n_kv_heads;
-    if ((size_t)(G + 1) * ctx->dec_max_cap * sizeof(float) > 200 * 1024) return CAKE_ERR_CAPACITY;
   }
   const int32_t rc = launch_decode_begin(ctx, ptrs, k_cache, v_cache, row_offsets_out, st);
   if (rc != CAKE_OK) return rc;

@@ -167,6 +167,7 @@ struct cake_ctx {
   int64_t* d_dec_off;             // [max_requests*L + 1] decode row offsets
   int64_t* d_dec_packed_off;      // [max_requests*L + 1] packed row offsets (set-up scratch)
   float* d_dec_score;             // stored eviction score of every slot
+  float* d_dec_tmp;               // [H_kv][tokens + requests][G + 1]: work area of decode heads too large for shared memory
   int32_t* d_dec_pos;             // token position of every slot (-1: free)
   int32_t* d_dec_order;           // per head: rank in ascending position -> slot
   int4* d_dec_meta;               // [max_lists] (len, free slot, next position, frozen budget)

@@ -14,12 +14,15 @@
 // Rows never move: the order of a head's entries by position is kept as a list of slots.
 #include "cake_internal.cuh"
 
+#include <algorithm>
+
 #include <math_constants.h>
 
 namespace cake {
 namespace {
 
-constexpr int DEC_THREADS = 256;
+constexpr int DEC_THREADS = 512;
+constexpr int DEC_ROWS = 4;       // cache rows a half-warp has in flight in the logit loop
 
 __device__ __forceinline__ float key_to_float(uint32_t key) {
   const uint32_t b = (key & 0x80000000u) ? (key & 0x7FFFFFFFu) : ~key;
@@ -92,6 +95,10 @@ struct DecodeArgs {
   int32_t* order;
   int4* meta;              // (len, free slot, next position, frozen budget)
   int32_t* status;
+  float* tmp;              // per (head, request) work area for heads beyond the shared-memory plan
+  const ReqInfo* reqs;
+  int64_t T;               // tokens of the batch
+  int n_req;
   int layer, L, Hq, Hkv, d, Sw, kp, pool_mode, update_mode, smem_cap;
   float scale2;
 };
@@ -99,6 +106,21 @@ struct DecodeArgs {
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// A lane's share of a row (up to 32 bytes held as four 8-byte words) as eight floats; elements
+// beyond the share are zero because the words beyond it are.
+template <typename T> __device__ __forceinline__ void unpack_row(const uint2 (&w)[4], float (&out)[8]);
+template <> __device__ __forceinline__ void unpack_row<float>(const uint2 (&w)[4], float (&out)[8]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { out[2 * i] = __uint_as_float(w[i].x); out[2 * i + 1] = __uint_as_float(w[i].y); }
+}
+template <> __device__ __forceinline__ void unpack_row<__nv_bfloat16>(const uint2 (&w)[4], float (&out)[8]) {
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    out[4 * i] = __uint_as_float(w[i].x << 16);     out[4 * i + 1] = __uint_as_float(w[i].x & 0xFFFF0000u);
+    out[4 * i + 2] = __uint_as_float(w[i].y << 16); out[4 * i + 3] = __uint_as_float(w[i].y & 0xFFFF0000u);
+  }
+}
 
 // (value, index) argmin with the tie rule of the eviction: the lowest score goes, among equal
 // scores the highest rank (= the highest token position).
@@ -123,12 +145,12 @@ decode_step_kernel(const DecodeArgs A) {
   const int len = mt.x, fre = mt.y, next_pos = mt.z, budget = mt.w;
   const int cap = len + 1;
   const int64_t base = A.dec_off[blk] + (int64_t)g * cap;
-  if (cap > A.smem_cap) {                            // does not fit the shared-memory plan
-    if (threadIdx.x == 0) atomicCAS(A.status, 0, CAKE_ERR_CAPACITY);
-    return;
-  }
-  float* p = sh;                                     // [G][cap]
-  float* abar = sh + (size_t)G * cap;                // [cap]
+  // A head beyond the shared-memory plan works in global memory: its (G + 1) * cap floats lie
+  // at the request's token offset of a [H_kv][tokens + requests] area (cap <= N + 1).
+  float* p = cap <= A.smem_cap                       // [G][cap]
+                 ? sh
+                 : A.tmp + (size_t)(G + 1) * ((size_t)g * (size_t)(A.T + A.n_req) + (size_t)A.reqs[req].cu + req);
+  float* abar = p + (size_t)G * cap;                 // [cap]
   T* kc = reinterpret_cast<T*>(A.k_cache) + (size_t)base * A.d;
   T* vc = reinterpret_cast<T*>(A.v_cache) + (size_t)base * A.d;
   const T* kn = reinterpret_cast<const T*>(A.k_new) + ((size_t)req * A.Hkv + g) * A.d;
@@ -152,29 +174,40 @@ decode_step_kernel(const DecodeArgs A) {
     for (int e = 0; e < 8; ++e)
       qv[h][e] = e < per ? to_f32(reinterpret_cast<const T*>(A.q_new)[((size_t)req * A.Hq + g * G + h) * A.d +
                                                                      l16 * per + e]) : 0.f;
-  for (int s0 = warp * 2; s0 < cap; s0 += (DEC_THREADS / 32) * 2) {
-    const int s = s0 + sub;
-    float kv[8];
+  // a lane's share of a row is 8, 16 or 32 bytes: 8-byte loads, DEC_ROWS rows in flight per half-warp
+  const int n8 = per * (int)sizeof(T) / 8;
+  constexpr int kStep = (DEC_THREADS / 32) * 2;
+  for (int s0 = warp * 2; s0 < cap; s0 += kStep * DEC_ROWS) {
+    uint2 raw[DEC_ROWS][4];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      kv[e] = 0.f;
-      if (s < cap && e < per)
-        kv[e] = s == fre ? to_f32(kn[l16 * per + e]) : to_f32(kc[(size_t)s * A.d + l16 * per + e]);
+    for (int u = 0; u < DEC_ROWS; ++u) {
+      const int s = s0 + u * kStep + sub;
+      const T* row = s == fre ? kn : kc + (size_t)s * A.d;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        raw[u][i] = (s < cap && i < n8) ? reinterpret_cast<const uint2*>(row + l16 * per)[i] : make_uint2(0u, 0u);
     }
 #pragma unroll
-    for (int h = 0; h < G; ++h) {
-      float acc = 0.f;
+    for (int u = 0; u < DEC_ROWS; ++u) {
+      const int s = s0 + u * kStep + sub;
+      float kv[8];
+      unpack_row<T>(raw[u], kv);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc = fmaf(qv[h][e], kv[e], acc);
+      for (int h = 0; h < G; ++h) {
+        float acc = 0.f;
 #pragma unroll
-      for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      if (l16 == 0 && s < cap) p[(size_t)h * cap + s] = acc * A.scale2;
+        for (int e = 0; e < 8; ++e) acc = fmaf(qv[h][e], kv[e], acc);
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (l16 == 0 && s < cap) p[(size_t)h * cap + s] = acc * A.scale2;
+      }
     }
   }
   __syncthreads();
   // 3. softmax per head over all cap slots (base 2)
   for (int h = 0; h < G; ++h) {
     float m = -CUDART_INF_F;
+#pragma unroll 4
     for (int s = threadIdx.x; s < cap; s += DEC_THREADS) m = fmaxf(m, p[(size_t)h * cap + s]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
@@ -184,6 +217,7 @@ decode_step_kernel(const DecodeArgs A) {
     for (int w = 1; w < DEC_THREADS / 32; ++w) m = fmaxf(m, red_v[w]);
     __syncthreads();
     float z = 0.f;
+#pragma unroll 4
     for (int s = threadIdx.x; s < cap; s += DEC_THREADS) {
       const float e = exp2f(p[(size_t)h * cap + s] - m);
       p[(size_t)h * cap + s] = e;
@@ -204,6 +238,7 @@ decode_step_kernel(const DecodeArgs A) {
   // 4. group-mean observed attention by rank (ascending position), pooling, score update
   const int n_obs = cap - A.Sw;                      // entries outside the recent window
   const int n_old = len - A.Sw;                      // of which these already carry a score
+#pragma unroll 4
   for (int r = threadIdx.x; r < n_obs; r += DEC_THREADS) {
     const int s = A.order[base + r];
     float a = 0.f;
@@ -215,6 +250,7 @@ decode_step_kernel(const DecodeArgs A) {
   const int rad = A.kp >> 1;
   float worst = CUDART_INF_F;
   int worst_r = -1;
+#pragma unroll 2
   for (int r = threadIdx.x; r < n_obs; r += DEC_THREADS) {
     const int lo = max(0, r - rad), hi = min(n_obs, r + rad + 1);
     float v = abar[lo];
@@ -256,11 +292,20 @@ decode_step_kernel(const DecodeArgs A) {
   // ranks after the evicted one move down by one; its slot becomes the free one
   const int ev_slot = A.order[base + ev];
   __syncthreads();
-  for (int r0 = ev; r0 < cap - 1; r0 += DEC_THREADS) {
-    const int r = r0 + threadIdx.x;
-    const int nxt = r < cap - 1 ? A.order[base + r + 1] : 0;
+  for (int r0 = ev; r0 < cap - 1; r0 += DEC_THREADS * 4) {       // four batches per round trip
+    int nxt[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int r = r0 + u * DEC_THREADS + threadIdx.x;
+      nxt[u] = r < cap - 1 ? A.order[base + r + 1] : 0;
+    }
     __syncthreads();
-    if (r < cap - 1) A.order[base + r] = nxt;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int r = r0 + u * DEC_THREADS + threadIdx.x;
+      if (r < cap - 1) A.order[base + r] = nxt[u];
+    }
+    __syncthreads();                                 // the next round reads beyond what this one wrote, but keep rounds apart
   }
   if (threadIdx.x == 0) {
     A.order[base + cap - 1] = ev_slot;
@@ -384,11 +429,13 @@ int32_t launch_decode_step(cake_ctx* ctx, int32_t layer, const void* q_new, cons
   A.layer = layer; A.L = c.n_layers; A.Hq = c.n_q_heads; A.Hkv = c.n_kv_heads; A.d = c.head_dim;
   A.Sw = c.window; A.kp = c.pool_kernel; A.pool_mode = c.pool_mode; A.update_mode = ctx->dec_update_mode;
   A.scale2 = 1.4426950408889634f / sqrtf((float)c.head_dim);
-  // shared memory: (G + 1) floats per slot; the largest head of the batch decides
-  const int64_t cap = ctx->dec_max_cap;
+  // shared memory: (G + 1) floats per slot, sized for the largest head of the batch up to the
+  // 200 KB the kernel may take; larger heads use the context's work area in global memory
+  const int64_t limit = (200 * 1024) / ((int64_t)(G + 1) * (int64_t)sizeof(float));
+  const int64_t cap = std::min<int64_t>(ctx->dec_max_cap, limit);
   const size_t smem = (size_t)(G + 1) * cap * sizeof(float);
-  if (smem > 200 * 1024) return CAKE_ERR_CAPACITY;
   A.smem_cap = (int)cap;
+  A.tmp = ctx->d_dec_tmp; A.reqs = ctx->d_req; A.T = ctx->total_tokens; A.n_req = ctx->n_req;
   const dim3 grid(c.n_kv_heads, ctx->n_req);
   const cudaError_t e = c.dtype == CAKE_DTYPE_FP32
                             ? launch_step<float>(ctx->device, G, grid, smem, st, A)

@@ -122,6 +122,14 @@ def test_decode_other_update_readings(mode):
     run_decode(w, steps=24, update_mode=mode)
 
 
+def test_decode_head_larger_than_shared_memory():
+    """G = 8 leaves the step kernel 5688 slots of shared memory per head; a head of about 6500
+    slots works in the context's global work area instead and must give the same results."""
+    w = synth.scaled(synth.workload(3), n_layers=1, n_q_heads=8, n_kv_heads=1, seq_lens=(7000, 400),
+                     total_budget=6500, window=16)
+    run_decode(w, steps=3)
+
+
 def test_decode_requires_a_finished_prefill():
     w = synth.scaled(synth.workload(1), n_layers=2, seq_lens=(100,), total_budget=2 * 30)
     qs, ks, vs = harness.device_inputs(w)
