@@ -15,6 +15,9 @@
 #include "cake_internal.cuh"
 
 #include <algorithm>
+#include <cstdlib>
+
+#include <cooperative_groups.h>
 
 #include <math_constants.h>
 
@@ -22,6 +25,8 @@ namespace cake {
 namespace {
 
 constexpr int DEC_THREADS = 512;
+constexpr int DEC_CLUSTER = 8;    // CTAs that share a head in the cluster form of the step kernel
+constexpr int DEC_CLUSTER_MIN_CAP = 512;   // smaller heads stay on one CTA
 constexpr int DEC_ROWS = 4;       // cache rows a half-warp has in flight in the logit loop
 
 __device__ __forceinline__ float key_to_float(uint32_t key) {
@@ -314,6 +319,232 @@ decode_step_kernel(const DecodeArgs A) {
   }
 }
 
+// The same step with a head spread over a thread-block cluster of DEC_CLUSTER CTAs: the head's
+// slots (logits, softmax) and then its ranks (pooling, score update, list shift) are cut into
+// DEC_CLUSTER contiguous parts, the per-head maxima, sums and the eviction candidate are exchanged
+// through distributed shared memory, and the group-mean attention passes from slot order to rank
+// order through the context's work area.  Every cluster barrier is reached by all CTAs of the
+// cluster: what decides the control flow (cap, the evicted rank) is the same in all of them.
+// Dynamic shared memory: G * part floats (logits by slot), reused for the pooled window and the
+// list shift.
+template <typename T, int G>
+__global__ void __launch_bounds__(DEC_THREADS)
+decode_step_cluster_kernel(const DecodeArgs A) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  extern __shared__ float sh[];
+  __shared__ float red_v[DEC_THREADS / 32];
+  __shared__ int red_i[DEC_THREADS / 32];
+  __shared__ float x_m[G], x_z[G];                   // this CTA's partial maximum / sum per head
+  __shared__ float x_worst;                          // this CTA's eviction candidate
+  __shared__ int x_worst_r;
+  __shared__ float s_m[G], s_z[G];
+  const int crank = (int)cluster.block_rank();
+  const int g = blockIdx.x / DEC_CLUSTER, req = blockIdx.y;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int blk = req * A.L + A.layer;
+  const size_t lid = (size_t)blk * A.Hkv + g;
+  const int4 mt = A.meta[lid];
+  const int len = mt.x, fre = mt.y, next_pos = mt.z, budget = mt.w;
+  const int cap = len + 1;
+  const int64_t base = A.dec_off[blk] + (int64_t)g * cap;
+  const int part = (cap + DEC_CLUSTER - 1) / DEC_CLUSTER;
+  const int s_lo = min(cap, crank * part), s_hi = min(cap, s_lo + part);
+  float* p = sh;                                     // [G][part], slot s at s - s_lo
+  float* aslot = A.tmp + (size_t)(G + 1) * ((size_t)g * (size_t)(A.T + A.n_req) + (size_t)A.reqs[req].cu + req);
+  T* kc = reinterpret_cast<T*>(A.k_cache) + (size_t)base * A.d;
+  T* vc = reinterpret_cast<T*>(A.v_cache) + (size_t)base * A.d;
+  const T* kn = reinterpret_cast<const T*>(A.k_new) + ((size_t)req * A.Hkv + g) * A.d;
+  const T* vn = reinterpret_cast<const T*>(A.v_new) + ((size_t)req * A.Hkv + g) * A.d;
+  // 1. the new token takes the free slot and the last rank (first CTA of the cluster)
+  if (crank == 0) {
+    for (int e = threadIdx.x; e < A.d; e += DEC_THREADS) {
+      kc[(size_t)fre * A.d + e] = kn[e];
+      vc[(size_t)fre * A.d + e] = vn[e];
+    }
+    if (threadIdx.x == 0) {
+      A.order[base + len] = fre;
+      A.pos[base + fre] = next_pos;
+    }
+  }
+  // 2. logits of the G query heads against this CTA's slots
+  const int sub = lane >> 4, l16 = lane & 15;
+  const int per = A.d / 16;
+  float qv[G][8];
+#pragma unroll
+  for (int h = 0; h < G; ++h)
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+      qv[h][e] = e < per ? to_f32(reinterpret_cast<const T*>(A.q_new)[((size_t)req * A.Hq + g * G + h) * A.d +
+                                                                     l16 * per + e]) : 0.f;
+  const int n8 = per * (int)sizeof(T) / 8;
+  constexpr int kStep = (DEC_THREADS / 32) * 2;
+  for (int s0 = s_lo + warp * 2; s0 < s_hi; s0 += kStep * DEC_ROWS) {
+    uint2 raw[DEC_ROWS][4];
+#pragma unroll
+    for (int u = 0; u < DEC_ROWS; ++u) {
+      const int s = s0 + u * kStep + sub;
+      const T* row = s == fre ? kn : kc + (size_t)s * A.d;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        raw[u][i] = (s < s_hi && i < n8) ? reinterpret_cast<const uint2*>(row + l16 * per)[i] : make_uint2(0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < DEC_ROWS; ++u) {
+      const int s = s0 + u * kStep + sub;
+      float kv[8];
+      unpack_row<T>(raw[u], kv);
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        float acc = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc = fmaf(qv[h][e], kv[e], acc);
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (l16 == 0 && s < s_hi) p[(size_t)h * part + (s - s_lo)] = acc * A.scale2;
+      }
+    }
+  }
+  __syncthreads();
+  // 3. softmax per head over all cap slots (base 2): partial maxima, then partial sums, each
+  //    combined over the cluster in rank order
+  const int n_loc = s_hi - s_lo;
+  for (int h = 0; h < G; ++h) {
+    float m = -CUDART_INF_F;
+    for (int i = threadIdx.x; i < n_loc; i += DEC_THREADS) m = fmaxf(m, p[(size_t)h * part + i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) red_v[warp] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float t = red_v[0];
+      for (int w = 1; w < DEC_THREADS / 32; ++w) t = fmaxf(t, red_v[w]);
+      x_m[h] = t;
+    }
+    __syncthreads();
+  }
+  cluster.sync();
+  if (threadIdx.x < G) {
+    float t = -CUDART_INF_F;
+    for (int c = 0; c < DEC_CLUSTER; ++c) t = fmaxf(t, *cluster.map_shared_rank(&x_m[threadIdx.x], c));
+    s_m[threadIdx.x] = t;
+  }
+  __syncthreads();
+  for (int h = 0; h < G; ++h) {
+    const float m = s_m[h];
+    float z = 0.f;
+    for (int i = threadIdx.x; i < n_loc; i += DEC_THREADS) {
+      const float e = exp2f(p[(size_t)h * part + i] - m);
+      p[(size_t)h * part + i] = e;
+      z += e;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    if (lane == 0) red_v[warp] = z;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float t = 0.f;
+      for (int w = 0; w < DEC_THREADS / 32; ++w) t += red_v[w];
+      x_z[h] = t;
+    }
+    __syncthreads();
+  }
+  cluster.sync();
+  if (threadIdx.x < G) {
+    float t = 0.f;
+    for (int c = 0; c < DEC_CLUSTER; ++c) t += *cluster.map_shared_rank(&x_z[threadIdx.x], c);
+    s_z[threadIdx.x] = t;
+  }
+  __syncthreads();
+  // 4. group-mean attention of this CTA's slots into the work area (by slot)
+  {
+    float inv_z[G];
+#pragma unroll
+    for (int h = 0; h < G; ++h) inv_z[h] = s_z[h];
+    for (int i = threadIdx.x; i < n_loc; i += DEC_THREADS) {
+      float a = 0.f;
+#pragma unroll
+      for (int h = 0; h < G; ++h) a += p[(size_t)h * part + i] / inv_z[h];
+      aslot[s_lo + i] = a * (1.f / (float)G);
+    }
+  }
+  cluster.sync();                                    // every slot's value is written; sh is free
+  // 5. this CTA's ranks: pooling along the rank order, score update, eviction candidate
+  const int n_obs = cap - A.Sw;                      // entries outside the recent window
+  const int n_old = len - A.Sw;                      // of which these already carry a score
+  const int rad = A.kp >> 1;
+  const int rpart = (n_obs + DEC_CLUSTER - 1) / DEC_CLUSTER;
+  const int r_lo = min(n_obs, crank * rpart), r_hi = min(n_obs, r_lo + rpart);
+  const int w_lo = max(0, r_lo - rad), w_hi = min(n_obs, r_hi + rad);
+  float* abar = sh;                                  // ranks w_lo .. w_hi - 1
+#pragma unroll 4
+  for (int i = threadIdx.x; i < w_hi - w_lo; i += DEC_THREADS) abar[i] = aslot[A.order[base + w_lo + i]];
+  __syncthreads();
+  float worst = CUDART_INF_F;
+  int worst_r = -1;
+#pragma unroll 2
+  for (int r = r_lo + threadIdx.x; r < r_hi; r += DEC_THREADS) {
+    const int lo = max(0, r - rad), hi = min(n_obs, r + rad + 1);
+    float v = abar[lo - w_lo];
+    for (int x = lo + 1; x < hi; ++x) v = A.pool_mode == CAKE_POOL_MAX ? fmaxf(v, abar[x - w_lo]) : v + abar[x - w_lo];
+    if (A.pool_mode != CAKE_POOL_MAX) v /= (float)A.kp;
+    const int s = A.order[base + r];
+    float sc = v;
+    if (r < n_old) {
+      const float old = A.score[base + s];
+      sc = A.update_mode == CAKE_DECODE_ADD ? old + v : A.update_mode == CAKE_DECODE_MAX ? fmaxf(old, v) : v;
+    }
+    A.score[base + s] = sc;
+    worse_of(worst, worst_r, sc, r);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, worst, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, worst_r, o);
+    if (oi >= 0 && (worst_r < 0 || ov < worst || (ov == worst && oi > worst_r))) { worst = ov; worst_r = oi; }
+  }
+  if (lane == 0) { red_v[warp] = worst; red_i[warp] = worst_r; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float bv = CUDART_INF_F;
+    int bi = -1;
+    for (int w = 0; w < DEC_THREADS / 32; ++w)
+      if (red_i[w] >= 0 && (bi < 0 || red_v[w] < bv || (red_v[w] == bv && red_i[w] > bi))) { bv = red_v[w]; bi = red_i[w]; }
+    x_worst = bv;
+    x_worst_r = bi;
+  }
+  cluster.sync();
+  int ev = -1;
+  if (n_obs > budget) {
+    float bv = CUDART_INF_F;
+    for (int c = 0; c < DEC_CLUSTER; ++c) {
+      const float cv = *cluster.map_shared_rank(&x_worst, c);
+      const int ci = *cluster.map_shared_rank(&x_worst_r, c);
+      if (ci >= 0 && (ev < 0 || cv < bv || (cv == bv && ci > ev))) { bv = cv; ev = ci; }
+    }
+  }
+  if (ev < 0) {                                      // below the budget: the cache would have to grow
+    if (crank == 0 && threadIdx.x == 0) atomicCAS(A.status, 0, CAKE_ERR_CAPACITY);
+    cluster.sync();                                  // nobody leaves while its candidate may still be read
+    return;
+  }
+  // 6. ranks after the evicted one move down by one; its slot becomes the free one.  Every CTA
+  //    reads the successors of its part of the list, the cluster meets, then it writes them.
+  const int ev_slot = A.order[base + ev];
+  const int m_lo = max(ev, min(cap - 1, crank * part)), m_hi = max(m_lo, min(cap - 1, crank * part + part));
+  int* nxt = reinterpret_cast<int*>(sh);
+#pragma unroll 4
+  for (int i = threadIdx.x; i < m_hi - m_lo; i += DEC_THREADS) nxt[i] = A.order[base + m_lo + i + 1];
+  cluster.sync();
+#pragma unroll 4
+  for (int i = threadIdx.x; i < m_hi - m_lo; i += DEC_THREADS) A.order[base + m_lo + i] = nxt[i];
+  if (crank == 0 && threadIdx.x == 0) {
+    A.order[base + cap - 1] = ev_slot;
+    A.pos[base + ev_slot] = -1;
+    A.meta[lid] = make_int4(len, ev_slot, next_pos + 1, budget);
+  }
+}
+
 // Entries of one (request, layer) in ascending position: positions, scores (window entries 0),
 // slots.  One CTA per head.
 __global__ void decode_read_state(const int64_t* __restrict__ dec_off, const float* __restrict__ score,
@@ -359,6 +590,44 @@ decode_gather(LayerPtrs ptrs, const int64_t* __restrict__ packed_off, const int6
     const size_t drow = (size_t)(dec_off[lo] + (int64_t)g * (len + 1) + idx) * cpr + chunk;
     k_out[drow] = reinterpret_cast<const uint4*>(ptrs.k[l])[srow];
     v_out[drow] = reinterpret_cast<const uint4*>(ptrs.v[l])[srow];
+  }
+}
+
+template <typename T, int G>
+cudaError_t launch_step_cluster_g(dim3 grid, size_t smem, cudaStream_t st, const DecodeArgs& A) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid.x * DEC_CLUSTER, grid.y, 1);
+  cfg.blockDim = dim3(DEC_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = DEC_CLUSTER;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_step_cluster_kernel<T, G>, A);
+}
+
+template <typename T>
+cudaError_t launch_step_cluster(int device, int G, dim3 grid, size_t smem, cudaStream_t st, const DecodeArgs& A) {
+  static PerDeviceOnce attr;
+  if (attr.need(device)) {
+    cudaError_t e = cudaSuccess;
+#define CAKE_DEC_ATTR(GG) \
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_step_cluster_kernel<T, GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
+    CAKE_DEC_ATTR(1); CAKE_DEC_ATTR(2); CAKE_DEC_ATTR(4); CAKE_DEC_ATTR(8);
+#undef CAKE_DEC_ATTR
+    if (e != cudaSuccess) return e;
+    attr.mark(device);
+  }
+  switch (G) {
+    case 1: return launch_step_cluster_g<T, 1>(grid, smem, st, A);
+    case 2: return launch_step_cluster_g<T, 2>(grid, smem, st, A);
+    case 4: return launch_step_cluster_g<T, 4>(grid, smem, st, A);
+    case 8: return launch_step_cluster_g<T, 8>(grid, smem, st, A);
+    default: return cudaErrorInvalidValue;
   }
 }
 
@@ -437,9 +706,20 @@ int32_t launch_decode_step(cake_ctx* ctx, int32_t layer, const void* q_new, cons
   A.smem_cap = (int)cap;
   A.tmp = ctx->d_dec_tmp; A.reqs = ctx->d_req; A.T = ctx->total_tokens; A.n_req = ctx->n_req;
   const dim3 grid(c.n_kv_heads, ctx->n_req);
-  const cudaError_t e = c.dtype == CAKE_DTYPE_FP32
-                            ? launch_step<float>(ctx->device, G, grid, smem, st, A)
-                            : launch_step<__nv_bfloat16>(ctx->device, G, grid, smem, st, A);
+  // Large heads are spread over a cluster of DEC_CLUSTER CTAs each (CAKE_DECODE_CLUSTER=0 keeps
+  // every head on one CTA): G floats per slot of a CTA's part, reused for the pooled window.
+  const int64_t part = (ctx->dec_max_cap + DEC_CLUSTER - 1) / DEC_CLUSTER;
+  const size_t smem_cl = ((size_t)G * part + (size_t)c.pool_kernel + 8) * sizeof(float);
+  const char* env = getenv("CAKE_DECODE_CLUSTER");
+  const bool use_cluster = ctx->dec_max_cap >= DEC_CLUSTER_MIN_CAP && smem_cl <= 200 * 1024 &&
+                           !(env && env[0] == '0');
+  cudaError_t e;
+  if (use_cluster)
+    e = c.dtype == CAKE_DTYPE_FP32 ? launch_step_cluster<float>(ctx->device, G, grid, smem_cl, st, A)
+                                   : launch_step_cluster<__nv_bfloat16>(ctx->device, G, grid, smem_cl, st, A);
+  else
+    e = c.dtype == CAKE_DTYPE_FP32 ? launch_step<float>(ctx->device, G, grid, smem, st, A)
+                                   : launch_step<__nv_bfloat16>(ctx->device, G, grid, smem, st, A);
   count_launch();
   return cuda_status(e);
 }

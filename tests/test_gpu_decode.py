@@ -122,12 +122,22 @@ def test_decode_other_update_readings(mode):
     run_decode(w, steps=24, update_mode=mode)
 
 
-def test_decode_head_larger_than_shared_memory():
-    """G = 8 leaves the step kernel 5688 slots of shared memory per head; a head of about 6500
-    slots works in the context's global work area instead and must give the same results."""
+@pytest.mark.parametrize("cluster", ["1", "0"])
+def test_decode_large_heads(monkeypatch, cluster):
+    """Heads of 512 slots or more are spread over a thread-block cluster; with that form switched
+    off a head beyond the 5688 slots that G = 8 leaves in shared memory works in the context's
+    global work area.  Both must match the oracle like the one-CTA form does."""
+    monkeypatch.setenv("CAKE_DECODE_CLUSTER", cluster)
     w = synth.scaled(synth.workload(3), n_layers=1, n_q_heads=8, n_kv_heads=1, seq_lens=(7000, 400),
                      total_budget=6500, window=16)
     run_decode(w, steps=3)
+
+
+def test_decode_cluster_form_over_many_steps():
+    w = synth.scaled(synth.workload(3), n_layers=2, n_q_heads=8, n_kv_heads=2, seq_lens=(2500, 700),
+                     total_budget=2 * 900)
+    ties = run_decode(w, steps=24)
+    assert ties <= 4
 
 
 def test_decode_requires_a_finished_prefill():
