@@ -22,9 +22,39 @@ template <> __device__ __forceinline__ float ld_f32<__nv_bfloat16>(const __nv_bf
   return __bfloat162float(*p);
 }
 
+// A lane's `per` (2 or 4) consecutive elements of a row in one load of 4, 8 or 16 bytes.
+template <typename T> __device__ __forceinline__ void ld_lane(const T* p, int per, float (&x)[4]);
+template <> __device__ __forceinline__ void ld_lane<float>(const float* p, int per, float (&x)[4]) {
+  if (per == 4) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+  } else {
+    const float2 v = *reinterpret_cast<const float2*>(p);
+    x[0] = v.x; x[1] = v.y; x[2] = 0.f; x[3] = 0.f;
+  }
+}
+template <> __device__ __forceinline__ void ld_lane<__nv_bfloat16>(const __nv_bfloat16* p, int per, float (&x)[4]) {
+  uint2 v = make_uint2(0u, 0u);
+  if (per == 4) v = *reinterpret_cast<const uint2*>(p);
+  else v.x = *reinterpret_cast<const uint32_t*>(p);
+  x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);
+  x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xFFFF0000u);
+}
+
 __device__ __forceinline__ uint32_t code4(float x, float zero, float scale) {
   const float q = rintf(__fdiv_rn(__fsub_rn(x, zero), scale));
   return (uint32_t)fminf(fmaxf(q, 0.f), 15.f);
+}
+// The same code from a multiplication by rcp = 1 / scale (rounded to nearest).  x * rcp is within
+// a few 1e-6 of the exact quotient (codes are at most 15), so it rounds to the same integer as the
+// IEEE quotient unless it lies that close to a half-integer; only then (and for non-finite
+// operands, which fail the comparison) the IEEE division decides.
+__device__ __forceinline__ uint32_t code4_rcp(float x, float zero, float scale, float rcp) {
+  const float dlt = __fsub_rn(x, zero);
+  const float q0 = __fmul_rn(dlt, rcp);
+  const float h = q0 - floorf(q0);
+  if (!(fabsf(h - 0.5f) >= 1e-4f)) return code4(x, zero, scale);
+  return (uint32_t)fminf(fmaxf(rintf(q0), 0.f), 15.f);
 }
 __device__ __forceinline__ float scale_of(float mn, float mx) {
   return mx > mn ? __fdiv_rn(__fsub_rn(mx, mn), 15.f) : 1.f;
@@ -57,39 +87,58 @@ quant_values(LayerPtrs ptrs, const int64_t* __restrict__ offsets, const int32_t*
   const int lanes_per_group = group / per;
   const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-  for (int64_t row = warp0; row < total; row += n_warps) {
-    int lo = 0, hi = nblk - 1;                       // last block with offset <= row
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (offsets[mid] <= row) lo = mid; else hi = mid - 1;
-    }
-    const int r = lo / L, l = lo - r * L;
-    const int len = budget[lo] + Sw;
-    const int g = (int)((row - offsets[lo]) / len);
-    const T* src = reinterpret_cast<const T*>(ptrs.v[l]) +
-                   ((size_t)g * T_tokens + reqs[r].cu + pos_packed[row]) * d + lane * per;
-    float x[4], mn = CUDART_INF_F, mx = -CUDART_INF_F;
+  // four rows per warp and round trip: their addresses first, then their values
+  for (int64_t row0 = warp0 * 4; row0 < total; row0 += n_warps * 4) {
+    const T* src[4];
+    float x[4][4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      x[e] = e < per ? ld_f32(src + e) : 0.f;
-      if (e < per) { mn = fminf(mn, x[e]); mx = fmaxf(mx, x[e]); }
+    for (int u = 0; u < 4; ++u) {
+      const int64_t row = row0 + u;
+      src[u] = nullptr;
+      if (row < total) {
+        int lo = 0, hi = nblk - 1;                   // last block with offset <= row
+        while (lo < hi) {
+          const int mid = (lo + hi + 1) >> 1;
+          if (offsets[mid] <= row) lo = mid; else hi = mid - 1;
+        }
+        const int r = lo / L, l = lo - r * L;
+        const int len = budget[lo] + Sw;
+        const int g = (int)((row - offsets[lo]) / len);
+        src[u] = reinterpret_cast<const T*>(ptrs.v[l]) +
+                 ((size_t)g * T_tokens + reqs[r].cu + pos_packed[row]) * d + lane * per;
+      }
     }
-    for (int o = 1; o < lanes_per_group; o <<= 1) {
-      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    }
-    const float sc = scale_of(mn, mx);
-    uint32_t packed = 0;
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
-      if (e < per) packed |= code4(x[e], mn, sc) << (4 * e);
-    uint8_t* dst = codes + (size_t)row * (d / 2) + lane * (per / 2);
-    dst[0] = (uint8_t)(packed & 0xFF);
-    if (per == 4) dst[1] = (uint8_t)(packed >> 8);
-    if (lane % lanes_per_group == 0) {
-      const size_t gi = (size_t)row * (d / group) + lane / lanes_per_group;
-      scale[gi] = sc;
-      zero[gi] = mn;
+    for (int u = 0; u < 4; ++u) {
+      x[u][0] = x[u][1] = x[u][2] = x[u][3] = 0.f;
+      if (src[u]) ld_lane<T>(src[u], per, x[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int64_t row = row0 + u;
+      if (row >= total) break;                       // uniform over the warp
+      float mn = CUDART_INF_F, mx = -CUDART_INF_F;
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (e < per) { mn = fminf(mn, x[u][e]); mx = fmaxf(mx, x[u][e]); }
+      for (int o = 1; o < lanes_per_group; o <<= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      }
+      const float sc = scale_of(mn, mx);
+      const float rc = __frcp_rn(sc);
+      uint32_t packed = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (e < per) packed |= code4_rcp(x[u][e], mn, sc, rc) << (4 * e);
+      uint8_t* dst = codes + (size_t)row * (d / 2) + lane * (per / 2);
+      if (per == 4) *reinterpret_cast<uint16_t*>(dst) = (uint16_t)packed;
+      else dst[0] = (uint8_t)(packed & 0xFF);
+      if (lane % lanes_per_group == 0) {
+        const size_t gi = (size_t)row * (d / group) + lane / lanes_per_group;
+        scale[gi] = sc;
+        zero[gi] = mn;
+      }
     }
   }
 }
@@ -118,20 +167,36 @@ __global__ void quant_keys(LayerPtrs ptrs, const int64_t* __restrict__ offsets,
     const int t0 = (int)(rel - (int64_t)g * gpb) * group, t1 = min(len, t0 + group);
     const int64_t row0 = offsets[lo] + (int64_t)g * len;
     const T* base = reinterpret_cast<const T*>(ptrs.k[l]) + ((size_t)g * T_tokens + reqs[r].cu) * d + c;
+    // eight rows per round trip: their positions first, then their values
     float mn = CUDART_INF_F, mx = -CUDART_INF_F;
-    for (int t = t0; t < t1; ++t) {
-      const float x = ld_f32(base + (size_t)pos_packed[row0 + t] * d);
-      mn = fminf(mn, x);
-      mx = fmaxf(mx, x);
+    for (int t = t0; t < t1; t += 8) {
+      int ps[8];
+      float xs[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) ps[u] = t + u < t1 ? pos_packed[row0 + t + u] : -1;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) xs[u] = ps[u] >= 0 ? ld_f32(base + (size_t)ps[u] * d) : 0.f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (ps[u] >= 0) { mn = fminf(mn, xs[u]); mx = fmaxf(mx, xs[u]); }
     }
     const float sc = scale_of(mn, mx);
+    const float rc = __frcp_rn(sc);
     scale[(size_t)gi * d + c] = sc;
     zero[(size_t)gi * d + c] = mn;
-    for (int t = t0; t < t1; ++t) {
-      const float x = ld_f32(base + (size_t)pos_packed[row0 + t] * d);
-      const uint32_t q = code4(x, mn, sc);
-      const uint32_t hi4 = __shfl_down_sync(0xffffffffu, q, 1);
-      if ((c & 1) == 0) codes[(size_t)(row0 + t) * (d / 2) + (c >> 1)] = (uint8_t)(q | (hi4 << 4));
+    for (int t = t0; t < t1; t += 8) {
+      int ps[8];
+      float xs[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) ps[u] = t + u < t1 ? pos_packed[row0 + t + u] : -1;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) xs[u] = ps[u] >= 0 ? ld_f32(base + (size_t)ps[u] * d) : 0.f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const uint32_t q = code4_rcp(xs[u], mn, sc, rc);  // every lane takes part in the shuffle
+        const uint32_t hi4 = __shfl_down_sync(0xffffffffu, q, 1);
+        if (ps[u] >= 0 && (c & 1) == 0) codes[(size_t)(row0 + t + u) * (d / 2) + (c >> 1)] = (uint8_t)(q | (hi4 << 4));
+      }
     }
   }
 }
